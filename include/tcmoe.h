@@ -1,0 +1,169 @@
+/*
+ * tcmoe - token-centric MoE layer for NVIDIA B200 (sm_100a): C ABI.
+ *
+ * The library computes one expert-parallel MoE layer as the paper states it
+ * (Sec. II-A): a gate picks `topk` experts per token, Dispatch moves the token
+ * to the expert groups ("GPUs" in the paper, logical partitions of one HBM
+ * here) that host them, every chosen expert runs its FFN (GEMM-1, GEMM-2), and
+ * Combine aggregates the `topk` outputs.  Symbols: T tokens, d hidden size,
+ * f expert FFN width, E experts, k = topk, G expert groups, m = E / G experts
+ * per group, P = T * k (token, expert) pairs, N_disp = number of distinct
+ * (token, group) pairs.
+ *
+ * Conventions for every entry point
+ *  - All tensor pointers are DEVICE pointers unless the name ends in `_host`.
+ *    The caller owns every buffer, including the workspace; the library never
+ *    allocates or frees device memory and keeps no pointer after a call.
+ *  - bf16 tensors are raw 16-bit patterns, row-major, rows contiguous.  Every
+ *    pointer must be 16-byte aligned; x, xg, o, y, w1, w3, w2 and the workspace
+ *    128-byte aligned.
+ *  - Calls only enqueue work on `stream` (a cudaStream_t passed as void*) and
+ *    never synchronise, except moe_status.  Data-dependent sizes (N_disp,
+ *    counts) stay on the device.
+ *  - Return value: 0 on success, a negative MOE_ERR_* when the host rejects the
+ *    call (nothing is launched then).  Conditions only the device can see go
+ *    to a status block at the start of the workspace, read with moe_status.
+ *  - The workspace must be zero-filled once before first use (or
+ *    moe_status_reset called on it).  Calls that share a workspace must be
+ *    ordered on one stream.
+ *  - There is no CPU fallback: without a CUDA device every compute entry point
+ *    returns MOE_ERR_CUDA.
+ */
+#ifndef TCMOE_H_
+#define TCMOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  MOE_OK = 0,
+  MOE_ERR_INVALID_ARG = -1,        /* null pointer, bad enum, inconsistent sizes          */
+  MOE_ERR_UNSUPPORTED_SHAPE = -2,  /* shape outside the limits listed at moe_shape_t      */
+  MOE_ERR_WORKSPACE_TOO_SMALL = -3,
+  MOE_ERR_MISALIGNED = -4,
+  MOE_ERR_CUDA = -5,               /* a CUDA runtime / driver call failed (incl. no GPU)  */
+  /* device-side codes, reported through moe_status()[0] */
+  MOE_DEV_TIMEOUT = 1,             /* a bounded wait inside a kernel expired              */
+  MOE_DEV_INDEX_OUT_OF_RANGE = 2   /* an expert index outside [0, E) was read             */
+};
+/* bits of moe_status()[5] */
+enum { MOE_WARN_NONFINITE_LOGIT = 1 };
+
+enum { MOE_SCORE_SOFTMAX = 0,      /* weights = softmax over the k selected keys          */
+       MOE_SCORE_SIGMOID = 1 };    /* weights = sigmoid(key) renormalised over the k      */
+enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1 }; /* default (0): gate weight applied in GEMM-2's
+                                            epilogue, Combine un-weighted (Sec. III-C)    */
+
+/* Shape of one layer.  Limits: 1 <= k <= min(E, 32); E <= 1024; E % G == 0;
+ * d % 8 == 0; f % 8 == 0; T >= 0; T * max(k, G) < 2^31. */
+typedef struct {
+  int32_t T, d, f, E, k, G;
+  int32_t score_fn;   /* MOE_SCORE_* */
+  int32_t flags;      /* MOE_FLAG_*  */
+} moe_shape_t;
+
+/* Dispatch layout: the software form of the paper's per-destination AL tables
+ * (Sec. III-D: algebraic index = token id -> layout index = row in a dense
+ * buffer) and TID table (Sec. IV-B).  All int32 device arrays, caller-allocated.
+ * Rows inside an expert / group are in ascending token order. */
+typedef struct {
+  int32_t* expert_counts;   /* [E]    rows per expert (the paper's nactive[expert])      */
+  int32_t* expert_offsets;  /* [E+1]  exclusive prefix sum, [E] = T*k                    */
+  int32_t* group_counts;    /* [G]    dispatched rows per group                          */
+  int32_t* group_offsets;   /* [G+1]  exclusive prefix sum, [G] = N_disp                 */
+  int32_t* pair_row;        /* [T*k]  expert-sorted row of pair p = t*k + j              */
+  int32_t* row_pair;        /* [T*k]  inverse of pair_row                                */
+  int32_t* al;              /* [G*T]  layout index of token t in group g, or -1          */
+  int32_t* disp_token;      /* [T*min(k,G)] token of dispatched row n; first N_disp used */
+  int32_t* row_src;         /* [T*k]  dispatched row feeding expert row r                */
+} moe_layout_t;
+
+/* Bytes of workspace that any entry point may need for this shape. */
+int moe_workspace_bytes(const moe_shape_t* shape, size_t* bytes);
+
+/* Zero the status block of a workspace (enqueued on `stream`). */
+int moe_status_reset(void* ws, void* stream);
+
+/* Copy the status block to the host: out[0] code (0 = ok, MOE_DEV_*), out[1]
+ * where (kernel id), out[2] detail, out[3] aux, out[4] abort flag, out[5]
+ * warning bits, out[6..7] reserved.  Synchronises `stream`. */
+int moe_status(const void* ws, int32_t out[8], void* stream);
+
+const char* moe_strerror(int code);
+
+/* Gate (Sec. II-A "selected by the gate network"): logits = x * w_gate in fp32;
+ * key = logit + bias (one fp32 add); the k largest keys per token, ordered by
+ * (key descending, expert index ascending), the lowest index winning ties;
+ * gate weights over the selected keys per shape->score_fn.
+ *   x          [T, d]  bf16
+ *   w_gate     [d, E]  fp32, or NULL: `logits` is then an INPUT
+ *   logit_bias NULL, or fp32 [E] (bias_row_stride = 0) or [T, E] (stride = E)
+ *   logits     [T, E]  fp32 out (raw, before the bias)
+ *   topk_idx   [T, k]  int32 out;  topk_w [T, k] fp32 out (sums to 1 per token) */
+int moe_route(const moe_shape_t* shape, const void* x, const float* w_gate,
+              const float* logit_bias, int64_t bias_row_stride,
+              float* logits, int32_t* topk_idx, float* topk_w,
+              void* ws, size_t ws_bytes, void* stream);
+
+/* Dispatch (Sec. II-A; Sec. III-D switch routing: group = expert / m, one
+ * replica per group trimmed to that group's targets; AL management).  Builds
+ * the layout from topk_idx (experts of a token must be distinct) and writes
+ * one copy of x[t] per DISTINCT group the token's experts live in:
+ *   xg[group_offsets[g] + al[g][t], :] = x[t, :].
+ *   xg  [T*min(k,G), d] bf16 capacity; may be NULL to build the layout only. */
+int moe_dispatch(const moe_shape_t* shape, const void* x, const int32_t* topk_idx,
+                 const moe_layout_t* layout, void* xg,
+                 void* ws, size_t ws_bytes, void* stream);
+
+/* Expert FFN (Sec. II-A GEMM-1 / GEMM-2; Sec. III-C: gate weight in GEMM-2's
+ * epilogue).  For expert e and each of its rows r (expert-sorted order):
+ *   a = xg[row_src[r]];  h = silu(a W1[e]) * (a W3[e]);  o[r] = w_r * (h W2[e])
+ * with w_r = topk_w[row_pair[r]] (or 1 with MOE_FLAG_WEIGHT_IN_COMBINE).
+ * bf16 operands, fp32 accumulation, h and o rounded to bf16.
+ *   w1, w3 [E, d, f] bf16;  w2 [E, f, d] bf16;  o [T*k, d] bf16 out. */
+int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t* layout,
+                   const float* topk_w, const void* w1, const void* w3, const void* w2,
+                   void* o, void* ws, size_t ws_bytes, void* stream);
+
+/* Combine (Sec. II-A aggregation; Sec. III-D reduction logic): for dispatched
+ * row n = (t, g), pg[n] = sum of token t's expert rows that live in group g
+ * (pre-reduction inside the group, ascending slot j); y[t] = sum over groups
+ * (ascending g) of the partial sums; fp32 accumulation, un-permuted to token
+ * order.  With MOE_FLAG_WEIGHT_IN_COMBINE rows are scaled by topk_w here.
+ *   o [T*k, d] bf16;  pg NULL or [N_disp, d] bf16 out;  y [T, d] bf16 out. */
+int moe_combine(const moe_shape_t* shape, const void* o, const moe_layout_t* layout,
+                const int32_t* topk_idx, const float* topk_w, void* pg, void* y,
+                void* ws, size_t ws_bytes, void* stream);
+
+/* Fused layer (Sec. IV token-centric kernel fusion): gate, layout, expert FFN
+ * fed straight from x (the dispatched copy is never written: the gather is
+ * GEMM-1's prologue) and combine, in one call.  logits, topk_idx, topk_w and
+ * layout are optional outputs (NULL: kept in the workspace). */
+int moe_layer(const moe_shape_t* shape, const void* x, const float* w_gate,
+              const float* logit_bias, int64_t bias_row_stride,
+              const void* w1, const void* w3, const void* w2, void* y,
+              float* logits, int32_t* topk_idx, float* topk_w, const moe_layout_t* layout,
+              void* ws, size_t ws_bytes, void* stream);
+
+/* moe_layer on HOST activations: copies x_host -> x_dev, runs moe_layer, copies
+ * y_dev -> y_host, all enqueued on `stream` (pinned host memory makes the copies
+ * asynchronous).  x_dev / y_dev are caller-owned device staging buffers
+ * [T, d] bf16; weights and workspace stay on the device. */
+int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, const float* w_gate,
+                   const float* logit_bias, int64_t bias_row_stride,
+                   const void* w1, const void* w3, const void* w2, void* y_dev, void* y_host,
+                   void* ws, size_t ws_bytes, void* stream);
+
+/* Byte offsets of named regions inside the workspace, for tests and profilers:
+ * out[0] status, out[1] h (GEMM-1 output [T*k, f] bf16), out[2] o scratch used
+ * by moe_layer, out[3] expert m-tile prefix [E+1] int32. */
+int moe_workspace_layout(const moe_shape_t* shape, size_t out[4]);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TCMOE_H_ */

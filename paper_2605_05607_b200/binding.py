@@ -1,0 +1,201 @@
+"""ctypes binding of libtcmoe.so: the same entry points as include/tcmoe.h.
+
+Argument marshalling only - every step of the path runs in the library's CUDA
+kernels.  PyTorch supplies device memory and streams.  There is no fallback:
+if the shared library is missing or cannot be loaded, importing a function from
+here raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from .synth import MoEConfig
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtcmoe.so")
+
+MOE_OK = 0
+MOE_ERR_INVALID_ARG = -1
+MOE_ERR_UNSUPPORTED_SHAPE = -2
+MOE_ERR_WORKSPACE_TOO_SMALL = -3
+MOE_ERR_MISALIGNED = -4
+MOE_ERR_CUDA = -5
+MOE_DEV_TIMEOUT = 1
+MOE_DEV_INDEX_OUT_OF_RANGE = 2
+MOE_WARN_NONFINITE_LOGIT = 1
+MOE_FLAG_WEIGHT_IN_COMBINE = 1
+
+EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "moe_status", "moe_strerror",
+           "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host")
+
+
+class MoEShape(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("T", "d", "f", "E", "k", "G", "score_fn", "flags")]
+
+
+class MoELayoutC(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_void_p) for n in
+                ("expert_counts", "expert_offsets", "group_counts", "group_offsets", "pair_row", "row_pair",
+                 "al", "disp_token", "row_src")]
+
+
+class MoEError(RuntimeError):
+    def __init__(self, fn: str, code: int):
+        self.code = code
+        super().__init__(f"{fn} failed: {code} ({strerror(code)})")
+
+
+_lib_handle = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the C-ABI library (built in-tree by paper_2605_05607_b200.build)."""
+    global _lib_handle
+    if _lib_handle is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2605_05607_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, sz = ctypes.c_void_p, ctypes.c_int64, ctypes.c_size_t
+        shp, lay = ctypes.POINTER(MoEShape), ctypes.POINTER(MoELayoutC)
+        L.moe_workspace_bytes.argtypes = [shp, ctypes.POINTER(sz)]
+        L.moe_workspace_layout.argtypes = [shp, ctypes.POINTER(sz)]
+        L.moe_status_reset.argtypes = [vp, vp]
+        L.moe_status.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), vp]
+        L.moe_strerror.argtypes = [ctypes.c_int]
+        L.moe_strerror.restype = ctypes.c_char_p
+        L.moe_route.argtypes = [shp, vp, vp, vp, i64, vp, vp, vp, vp, sz, vp]
+        L.moe_dispatch.argtypes = [shp, vp, vp, lay, vp, vp, sz, vp]
+        L.moe_expert_ffn.argtypes = [shp, vp, lay, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.moe_combine.argtypes = [shp, vp, lay, vp, vp, vp, vp, vp, sz, vp]
+        L.moe_layer.argtypes = [shp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, lay, vp, sz, vp]
+        L.moe_layer_host.argtypes = [shp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
+        for name in EXPORTS:
+            if name != "moe_strerror":
+                getattr(L, name).restype = ctypes.c_int
+        _lib_handle = L
+    return _lib_handle
+
+
+def make_shape(cfg: MoEConfig, flags: int = 0) -> MoEShape:
+    return MoEShape(cfg.T, cfg.d, cfg.f, cfg.E, cfg.k, cfg.G, cfg.score_fn, flags)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    if t is None:
+        return None
+    assert t.is_contiguous(), "tensors passed to the C ABI must be contiguous"
+    return t.data_ptr()
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream() if torch.cuda.is_available() else None
+    return None if stream is None else stream.cuda_stream
+
+
+def _check(fn: str, rc: int) -> None:
+    if rc != MOE_OK:
+        raise MoEError(fn, rc)
+
+
+def strerror(code: int) -> str:
+    return lib().moe_strerror(code).decode()
+
+
+@dataclass
+class Layout:
+    """Device int32 tensors of moe_layout_t."""
+    expert_counts: torch.Tensor
+    expert_offsets: torch.Tensor
+    group_counts: torch.Tensor
+    group_offsets: torch.Tensor
+    pair_row: torch.Tensor
+    row_pair: torch.Tensor
+    al: torch.Tensor
+    disp_token: torch.Tensor
+    row_src: torch.Tensor
+
+    def c(self) -> MoELayoutC:
+        return MoELayoutC(*[getattr(self, n).data_ptr() for n, _ in MoELayoutC._fields_])
+
+
+def alloc_layout(shape: MoEShape, device="cuda") -> Layout:
+    T, E, k, G = shape.T, shape.E, shape.k, shape.G
+    z = lambda n: torch.zeros(max(n, 4), dtype=torch.int32, device=device)
+    return Layout(z(E), z(E + 1), z(G), z(G + 1), z(T * k), z(T * k), z(G * T), z(T * min(k, G)), z(T * k))
+
+
+def moe_workspace_bytes(shape: MoEShape) -> int:
+    out = ctypes.c_size_t(0)
+    _check("moe_workspace_bytes", lib().moe_workspace_bytes(ctypes.byref(shape), ctypes.byref(out)))
+    return out.value
+
+
+def moe_workspace_layout(shape: MoEShape) -> dict:
+    out = (ctypes.c_size_t * 4)()
+    _check("moe_workspace_layout", lib().moe_workspace_layout(ctypes.byref(shape), out))
+    return {"status": out[0], "h": out[1], "o": out[2], "mt_prefix": out[3]}
+
+
+def alloc_workspace(shape: MoEShape, device="cuda") -> torch.Tensor:
+    """Zero-filled workspace (the status block must start at zero)."""
+    return torch.zeros(moe_workspace_bytes(shape), dtype=torch.uint8, device=device)
+
+
+def moe_status_reset(ws: torch.Tensor, stream=None) -> None:
+    _check("moe_status_reset", lib().moe_status_reset(_ptr(ws), _stream(stream)))
+
+
+def moe_status(ws: torch.Tensor, stream=None) -> list:
+    out = (ctypes.c_int32 * 8)()
+    _check("moe_status", lib().moe_status(_ptr(ws), out, _stream(stream)))
+    return list(out)
+
+
+def moe_route(shape, x, w_gate, logit_bias, logits, topk_idx, topk_w, ws, stream=None) -> None:
+    stride = 0 if logit_bias is None or logit_bias.dim() == 1 else shape.E
+    _check("moe_route", lib().moe_route(ctypes.byref(shape), _ptr(x), _ptr(w_gate), _ptr(logit_bias), stride,
+                                        _ptr(logits), _ptr(topk_idx), _ptr(topk_w), _ptr(ws), ws.numel(),
+                                        _stream(stream)))
+
+
+def moe_dispatch(shape, x, topk_idx, layout: Layout, xg, ws, stream=None) -> None:
+    c = layout.c()
+    _check("moe_dispatch", lib().moe_dispatch(ctypes.byref(shape), _ptr(x), _ptr(topk_idx), ctypes.byref(c),
+                                              _ptr(xg), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def moe_expert_ffn(shape, xg, layout: Layout, topk_w, w1, w3, w2, o, ws, stream=None) -> None:
+    c = layout.c()
+    _check("moe_expert_ffn", lib().moe_expert_ffn(ctypes.byref(shape), _ptr(xg), ctypes.byref(c), _ptr(topk_w),
+                                                  _ptr(w1), _ptr(w3), _ptr(w2), _ptr(o), _ptr(ws), ws.numel(),
+                                                  _stream(stream)))
+
+
+def moe_combine(shape, o, layout: Layout, topk_idx, topk_w, pg, y, ws, stream=None) -> None:
+    c = layout.c()
+    _check("moe_combine", lib().moe_combine(ctypes.byref(shape), _ptr(o), ctypes.byref(c), _ptr(topk_idx),
+                                            _ptr(topk_w), _ptr(pg), _ptr(y), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def moe_layer(shape, x, w_gate, logit_bias, w1, w3, w2, y, ws, logits=None, topk_idx=None, topk_w=None,
+              layout: Optional[Layout] = None, stream=None) -> None:
+    stride = 0 if logit_bias is None or logit_bias.dim() == 1 else shape.E
+    c = layout.c() if layout is not None else None
+    _check("moe_layer", lib().moe_layer(ctypes.byref(shape), _ptr(x), _ptr(w_gate), _ptr(logit_bias), stride,
+                                        _ptr(w1), _ptr(w3), _ptr(w2), _ptr(y), _ptr(logits), _ptr(topk_idx),
+                                        _ptr(topk_w), ctypes.byref(c) if c is not None else None, _ptr(ws),
+                                        ws.numel(), _stream(stream)))
+
+
+def moe_layer_host(shape, x_host, x_dev, w_gate, logit_bias, w1, w3, w2, y_dev, y_host, ws, stream=None) -> None:
+    stride = 0 if logit_bias is None or logit_bias.dim() == 1 else shape.E
+    _check("moe_layer_host", lib().moe_layer_host(ctypes.byref(shape), _ptr(x_host), _ptr(x_dev), _ptr(w_gate),
+                                                  _ptr(logit_bias), stride, _ptr(w1), _ptr(w3), _ptr(w2),
+                                                  _ptr(y_dev), _ptr(y_host), _ptr(ws), ws.numel(), _stream(stream)))

@@ -1,0 +1,347 @@
+// C ABI of the library: argument checks, workspace carving, stage sequencing.
+#include "../../include/tcmoe.h"
+
+#include "common.cuh"
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tcmoe {
+namespace {
+
+constexpr size_t ALIGN = 1024;
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Regions of the workspace, in order.  Every region starts on a 1 KiB boundary.
+struct WsPlan {
+  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, h, o, logits, topk_idx, topk_w;
+  size_t expert_counts, expert_offsets, group_counts, group_offsets, pair_row, row_pair, al, disp_token, row_src;
+  size_t total;
+  int W;
+};
+
+WsPlan plan(const moe_shape_t& s) {
+  WsPlan p{};
+  const size_t T = (size_t)s.T, E = (size_t)s.E, G = (size_t)s.G, k = (size_t)s.k;
+  const size_t P = T * k;
+  const size_t W = (T + 31) / 32;
+  const size_t kg = k < G ? k : G;
+  p.W = (int)W;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off = round_up(off + bytes, ALIGN);
+    return at;
+  };
+  p.status = take(64);
+  p.emask = off;  // emask and gmask must be adjacent (one memset clears both)
+  off += E * W * 4;
+  p.gmask = off;
+  off = round_up(off + G * W * 4, ALIGN);
+  p.eprefix = take(E * W * 4);
+  p.gprefix = take(G * W * 4);
+  p.mt_prefix = take((E + 1) * 4);
+  p.h = take(P * (size_t)s.f * 2);
+  p.o = take(P * (size_t)s.d * 2);
+  p.logits = take(T * E * 4);
+  p.topk_idx = take(P * 4);
+  p.topk_w = take(P * 4);
+  p.expert_counts = take(E * 4);
+  p.expert_offsets = take((E + 1) * 4);
+  p.group_counts = take(G * 4);
+  p.group_offsets = take((G + 1) * 4);
+  p.pair_row = take(P * 4);
+  p.row_pair = take(P * 4);
+  p.al = take(G * T * 4);
+  p.disp_token = take(T * kg * 4);
+  p.row_src = take(P * 4);
+  p.total = off;
+  return p;
+}
+
+int check_shape(const moe_shape_t* s) {
+  if (s == nullptr) return MOE_ERR_INVALID_ARG;
+  if (s->T < 0 || s->d <= 0 || s->f <= 0 || s->E <= 0 || s->k <= 0 || s->G <= 0) return MOE_ERR_INVALID_ARG;
+  if (s->score_fn != MOE_SCORE_SOFTMAX && s->score_fn != MOE_SCORE_SIGMOID) return MOE_ERR_INVALID_ARG;
+  if (s->flags & ~MOE_FLAG_WEIGHT_IN_COMBINE) return MOE_ERR_INVALID_ARG;
+  if (s->k > s->E || s->G > s->E || s->E % s->G != 0) return MOE_ERR_INVALID_ARG;
+  if (s->k > 32 || s->E > 1024 || s->d % 8 != 0 || s->f % 8 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
+  const long long kg = s->k > s->G ? s->k : s->G;
+  if ((long long)s->T * kg >= (1ll << 31)) return MOE_ERR_UNSUPPORTED_SHAPE;
+  return MOE_OK;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int check_ws(const moe_shape_t* s, const void* ws, size_t ws_bytes, WsPlan* out) {
+  if (ws == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!aligned(ws, 128)) return MOE_ERR_MISALIGNED;
+  *out = plan(*s);
+  if (ws_bytes < out->total) return MOE_ERR_WORKSPACE_TOO_SMALL;
+  return MOE_OK;
+}
+
+int check_layout(const moe_layout_t* L) {
+  if (L == nullptr) return MOE_ERR_INVALID_ARG;
+  const void* ptrs[9] = {L->expert_counts, L->expert_offsets, L->group_counts, L->group_offsets, L->pair_row,
+                         L->row_pair,      L->al,             L->disp_token,   L->row_src};
+  for (const void* p : ptrs) {
+    if (p == nullptr) return MOE_ERR_INVALID_ARG;
+    if (!aligned(p, 16)) return MOE_ERR_MISALIGNED;
+  }
+  return MOE_OK;
+}
+
+Shape to_shape(const moe_shape_t& s) { return Shape{s.T, s.d, s.f, s.E, s.k, s.G, s.score_fn, s.flags}; }
+Layout to_layout(const moe_layout_t& L) {
+  return Layout{L.expert_counts, L.expert_offsets, L.group_counts, L.group_offsets, L.pair_row,
+                L.row_pair,      L.al,             L.disp_token,   L.row_src};
+}
+template <typename T>
+T* at(void* ws, size_t off) { return reinterpret_cast<T*>(static_cast<uint8_t*>(ws) + off); }
+
+LayoutScratch scratch(void* ws, const WsPlan& p) {
+  LayoutScratch sc;
+  sc.emask = at<uint32_t>(ws, p.emask);
+  sc.gmask = at<uint32_t>(ws, p.gmask);
+  sc.eprefix = at<int32_t>(ws, p.eprefix);
+  sc.gprefix = at<int32_t>(ws, p.gprefix);
+  sc.mt_prefix = at<int32_t>(ws, p.mt_prefix);
+  sc.W = p.W;
+  return sc;
+}
+
+bool have_device() {
+  int n = 0;
+  return cudaGetDeviceCount(&n) == cudaSuccess && n > 0;
+}
+
+#define TCMOE_CUDA(expr)                     \
+  do {                                       \
+    if ((expr) != cudaSuccess) {             \
+      (void)cudaGetLastError();              \
+      return MOE_ERR_CUDA;                   \
+    }                                        \
+  } while (0)
+
+}  // namespace
+}  // namespace tcmoe
+
+using namespace tcmoe;
+
+extern "C" {
+
+int moe_workspace_bytes(const moe_shape_t* shape, size_t* bytes) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (bytes == nullptr) return MOE_ERR_INVALID_ARG;
+  *bytes = plan(*shape).total;
+  return MOE_OK;
+}
+
+int moe_workspace_layout(const moe_shape_t* shape, size_t out[4]) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (out == nullptr) return MOE_ERR_INVALID_ARG;
+  const WsPlan p = plan(*shape);
+  out[0] = p.status;
+  out[1] = p.h;
+  out[2] = p.o;
+  out[3] = p.mt_prefix;
+  return MOE_OK;
+}
+
+int moe_status_reset(void* ws, void* stream) {
+  if (ws == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!have_device()) return MOE_ERR_CUDA;
+  TCMOE_CUDA(cudaMemsetAsync(ws, 0, 64, static_cast<cudaStream_t>(stream)));
+  return MOE_OK;
+}
+
+int moe_status(const void* ws, int32_t out[8], void* stream) {
+  if (ws == nullptr || out == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!have_device()) return MOE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  TCMOE_CUDA(cudaMemcpyAsync(out, ws, 8 * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  TCMOE_CUDA(cudaStreamSynchronize(st));
+  return MOE_OK;
+}
+
+const char* moe_strerror(int code) {
+  switch (code) {
+    case MOE_OK: return "ok";
+    case MOE_ERR_INVALID_ARG: return "invalid argument";
+    case MOE_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+    case MOE_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case MOE_ERR_MISALIGNED: return "misaligned pointer";
+    case MOE_ERR_CUDA: return "CUDA error (or no CUDA device)";
+    case MOE_DEV_TIMEOUT: return "device: bounded wait expired";
+    case MOE_DEV_INDEX_OUT_OF_RANGE: return "device: expert index out of range";
+    default: return "unknown code";
+  }
+}
+
+int moe_route(const moe_shape_t* shape, const void* x, const float* w_gate, const float* logit_bias,
+              int64_t bias_row_stride, float* logits, int32_t* topk_idx, float* topk_w, void* ws, size_t ws_bytes,
+              void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (logits == nullptr || topk_idx == nullptr || topk_w == nullptr) return MOE_ERR_INVALID_ARG;
+  if (w_gate != nullptr && x == nullptr) return MOE_ERR_INVALID_ARG;
+  if (bias_row_stride != 0 && bias_row_stride != shape->E) return MOE_ERR_INVALID_ARG;
+  if (!aligned(x, 16) || !aligned(w_gate, 16) || !aligned(logits, 16) || !aligned(topk_idx, 16) ||
+      !aligned(topk_w, 16) || !aligned(logit_bias, 4))
+    return MOE_ERR_MISALIGNED;
+  WsPlan p;
+  if ((rc = check_ws(shape, ws, ws_bytes, &p)) != MOE_OK) return rc;
+  if (!have_device()) return MOE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Shape s = to_shape(*shape);
+  if (w_gate != nullptr) TCMOE_CUDA(launch_gate_logits(s, x, w_gate, logits, st));
+  TCMOE_CUDA(launch_topk(s, logits, logit_bias, bias_row_stride, topk_idx, topk_w, at<int32_t>(ws, p.status), st));
+  return MOE_OK;
+}
+
+int moe_dispatch(const moe_shape_t* shape, const void* x, const int32_t* topk_idx, const moe_layout_t* layout,
+                 void* xg, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (topk_idx == nullptr || (xg != nullptr && x == nullptr)) return MOE_ERR_INVALID_ARG;
+  if ((rc = check_layout(layout)) != MOE_OK) return rc;
+  if (!aligned(x, 128) || !aligned(xg, 128) || !aligned(topk_idx, 16)) return MOE_ERR_MISALIGNED;
+  WsPlan p;
+  if ((rc = check_ws(shape, ws, ws_bytes, &p)) != MOE_OK) return rc;
+  if (!have_device()) return MOE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Shape s = to_shape(*shape);
+  const Layout L = to_layout(*layout);
+  TCMOE_CUDA(launch_layout(s, topk_idx, L, scratch(ws, p), at<int32_t>(ws, p.status), st));
+  if (xg != nullptr) TCMOE_CUDA(launch_dispatch(s, x, L, xg, st));
+  return MOE_OK;
+}
+
+int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t* layout, const float* topk_w,
+                   const void* w1, const void* w3, const void* w2, void* o, void* ws, size_t ws_bytes,
+                   void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (xg == nullptr || w1 == nullptr || w3 == nullptr || w2 == nullptr || o == nullptr) return MOE_ERR_INVALID_ARG;
+  const bool in_combine = (shape->flags & MOE_FLAG_WEIGHT_IN_COMBINE) != 0;
+  if (!in_combine && topk_w == nullptr) return MOE_ERR_INVALID_ARG;
+  if ((rc = check_layout(layout)) != MOE_OK) return rc;
+  if (!aligned(xg, 128) || !aligned(w1, 128) || !aligned(w3, 128) || !aligned(w2, 128) || !aligned(o, 128) ||
+      !aligned(topk_w, 16))
+    return MOE_ERR_MISALIGNED;
+  WsPlan p;
+  if ((rc = check_ws(shape, ws, ws_bytes, &p)) != MOE_OK) return rc;
+  if (!have_device()) return MOE_ERR_CUDA;
+  FfnArgs a{};
+  a.a_src = xg;
+  a.gather_idx = layout->row_src;
+  a.gather_div = 1;
+  a.w1 = w1;
+  a.w3 = w3;
+  a.w2 = w2;
+  a.h = at<void>(ws, p.h);
+  a.o = o;
+  a.topk_w = in_combine ? nullptr : topk_w;
+  a.row_pair = layout->row_pair;
+  a.expert_offsets = layout->expert_offsets;
+  a.mt_prefix = at<int32_t>(ws, p.mt_prefix);
+  a.status = at<int32_t>(ws, p.status);
+  // rebuilt from the counts so that this call does not depend on what moe_dispatch left in ws
+  TCMOE_CUDA(launch_mt_prefix(to_shape(*shape), layout->expert_counts, at<int32_t>(ws, p.mt_prefix),
+                              static_cast<cudaStream_t>(stream)));
+  TCMOE_CUDA(launch_expert_ffn(to_shape(*shape), a, static_cast<cudaStream_t>(stream)));
+  return MOE_OK;
+}
+
+int moe_combine(const moe_shape_t* shape, const void* o, const moe_layout_t* layout, const int32_t* topk_idx,
+                const float* topk_w, void* pg, void* y, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (o == nullptr || y == nullptr || topk_idx == nullptr) return MOE_ERR_INVALID_ARG;
+  if ((shape->flags & MOE_FLAG_WEIGHT_IN_COMBINE) && topk_w == nullptr) return MOE_ERR_INVALID_ARG;
+  if ((rc = check_layout(layout)) != MOE_OK) return rc;
+  if (!aligned(o, 128) || !aligned(y, 128) || !aligned(pg, 128) || !aligned(topk_idx, 16) || !aligned(topk_w, 16))
+    return MOE_ERR_MISALIGNED;
+  WsPlan p;
+  if ((rc = check_ws(shape, ws, ws_bytes, &p)) != MOE_OK) return rc;
+  if (!have_device()) return MOE_ERR_CUDA;
+  TCMOE_CUDA(launch_combine(to_shape(*shape), o, to_layout(*layout), topk_idx, topk_w, pg, y,
+                            static_cast<cudaStream_t>(stream)));
+  return MOE_OK;
+}
+
+int moe_layer(const moe_shape_t* shape, const void* x, const float* w_gate, const float* logit_bias,
+              int64_t bias_row_stride, const void* w1, const void* w3, const void* w2, void* y, float* logits,
+              int32_t* topk_idx, float* topk_w, const moe_layout_t* layout, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (x == nullptr || w_gate == nullptr || w1 == nullptr || w3 == nullptr || w2 == nullptr || y == nullptr)
+    return MOE_ERR_INVALID_ARG;
+  if (bias_row_stride != 0 && bias_row_stride != shape->E) return MOE_ERR_INVALID_ARG;
+  if (layout != nullptr && (rc = check_layout(layout)) != MOE_OK) return rc;
+  if (!aligned(x, 128) || !aligned(w1, 128) || !aligned(w3, 128) || !aligned(w2, 128) || !aligned(y, 128) ||
+      !aligned(w_gate, 16) || !aligned(logits, 16) || !aligned(topk_idx, 16) || !aligned(topk_w, 16) ||
+      !aligned(logit_bias, 4))
+    return MOE_ERR_MISALIGNED;
+  WsPlan p;
+  if ((rc = check_ws(shape, ws, ws_bytes, &p)) != MOE_OK) return rc;
+  if (!have_device()) return MOE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const Shape s = to_shape(*shape);
+  int32_t* status = at<int32_t>(ws, p.status);
+  float* lg = logits != nullptr ? logits : at<float>(ws, p.logits);
+  int32_t* idx = topk_idx != nullptr ? topk_idx : at<int32_t>(ws, p.topk_idx);
+  float* tw = topk_w != nullptr ? topk_w : at<float>(ws, p.topk_w);
+  Layout L;
+  if (layout != nullptr) {
+    L = to_layout(*layout);
+  } else {
+    L = Layout{at<int32_t>(ws, p.expert_counts), at<int32_t>(ws, p.expert_offsets), at<int32_t>(ws, p.group_counts),
+               at<int32_t>(ws, p.group_offsets), at<int32_t>(ws, p.pair_row),       at<int32_t>(ws, p.row_pair),
+               at<int32_t>(ws, p.al),            at<int32_t>(ws, p.disp_token),     at<int32_t>(ws, p.row_src)};
+  }
+  // gate
+  TCMOE_CUDA(launch_gate_logits(s, x, w_gate, lg, st));
+  TCMOE_CUDA(launch_topk(s, lg, logit_bias, bias_row_stride, idx, tw, status, st));
+  // layout only: the dispatched copy xg is never written, GEMM-1 gathers token rows from x
+  TCMOE_CUDA(launch_layout(s, idx, L, scratch(ws, p), status, st));
+  FfnArgs a{};
+  a.a_src = x;
+  a.gather_idx = L.row_pair;   // token of expert row r = row_pair[r] / k
+  a.gather_div = s.k;
+  a.w1 = w1;
+  a.w3 = w3;
+  a.w2 = w2;
+  a.h = at<void>(ws, p.h);
+  a.o = at<void>(ws, p.o);
+  a.topk_w = (s.flags & MOE_FLAG_WEIGHT_IN_COMBINE) ? nullptr : tw;
+  a.row_pair = L.row_pair;
+  a.expert_offsets = L.expert_offsets;
+  a.mt_prefix = at<int32_t>(ws, p.mt_prefix);
+  a.status = status;
+  TCMOE_CUDA(launch_expert_ffn(s, a, st));
+  TCMOE_CUDA(launch_combine(s, a.o, L, idx, tw, nullptr, y, st));
+  return MOE_OK;
+}
+
+int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, const float* w_gate,
+                   const float* logit_bias, int64_t bias_row_stride, const void* w1, const void* w3, const void* w2,
+                   void* y_dev, void* y_host, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (x_host == nullptr || x_dev == nullptr || y_dev == nullptr || y_host == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!have_device()) return MOE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)shape->T * shape->d * 2;
+  if (bytes) TCMOE_CUDA(cudaMemcpyAsync(x_dev, x_host, bytes, cudaMemcpyHostToDevice, st));
+  rc = moe_layer(shape, x_dev, w_gate, logit_bias, bias_row_stride, w1, w3, w2, y_dev, nullptr, nullptr, nullptr,
+                 nullptr, ws, ws_bytes, stream);
+  if (rc != MOE_OK) return rc;
+  if (bytes) TCMOE_CUDA(cudaMemcpyAsync(y_host, y_dev, bytes, cudaMemcpyDeviceToHost, st));
+  return MOE_OK;
+}
+
+}  // extern "C"

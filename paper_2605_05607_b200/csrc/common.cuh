@@ -1,0 +1,72 @@
+// Internal declarations shared by the tcmoe translation units (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tcmoe {
+
+// ---- status block at the start of the workspace (16 x int32) --------------------------------
+enum StatusSlot { ST_CODE = 0, ST_WHERE = 1, ST_DETAIL = 2, ST_AUX = 3, ST_ABORT = 4, ST_WARN = 5 };
+enum KernelId { KID_TOPK = 1, KID_MASKS = 2, KID_FILL = 3, KID_DISPATCH = 4, KID_GEMM1 = 5, KID_GEMM2 = 6,
+                KID_COMBINE = 7, KID_GATE = 8 };
+constexpr int DEV_TIMEOUT = 1;
+constexpr int DEV_INDEX_OUT_OF_RANGE = 2;
+constexpr int WARN_NONFINITE_LOGIT = 1;
+
+__device__ __forceinline__ void report_error(int32_t* status, int code, int where, int detail, int aux) {
+  if (atomicCAS(&status[ST_CODE], 0, code) == 0) {
+    status[ST_WHERE] = where;
+    status[ST_DETAIL] = detail;
+    status[ST_AUX] = aux;
+  }
+}
+
+// ---- problem description passed to the launchers ---------------------------------------------
+struct Shape {
+  int T, d, f, E, k, G, score_fn, flags;
+};
+
+struct Layout {
+  int32_t *expert_counts, *expert_offsets, *group_counts, *group_offsets, *pair_row, *row_pair, *al,
+      *disp_token, *row_src;
+};
+
+// Scratch tables of the layout builder (inside the workspace).
+struct LayoutScratch {
+  uint32_t* emask;    // [E, W] bit t%32 of word t/32: token t selected expert e
+  uint32_t* gmask;    // [G, W] token t touches group g
+  int32_t* eprefix;   // [E, W] exclusive popcount prefix along the row
+  int32_t* gprefix;   // [G, W]
+  int32_t* mt_prefix; // [E+1]  exclusive prefix of 128-row tiles per expert
+  int W;
+};
+
+// route.cu
+cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gate, float* logits, cudaStream_t st);
+cudaError_t launch_topk(const Shape& s, const float* logits, const float* bias, int64_t bias_stride,
+                        int32_t* topk_idx, float* topk_w, int32_t* status, cudaStream_t st);
+// layout.cu
+cudaError_t launch_layout(const Shape& s, const int32_t* topk_idx, const Layout& L, const LayoutScratch& sc,
+                          int32_t* status, cudaStream_t st);
+cudaError_t launch_mt_prefix(const Shape& s, const int32_t* expert_counts, int32_t* mt_prefix, cudaStream_t st);
+cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void* xg, cudaStream_t st);
+cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
+                           const float* topk_w, void* pg, void* y, cudaStream_t st);
+// ffn.cu
+struct FfnArgs {
+  const void* a_src;          // GEMM-1 activations: xg (gather_div = 1) or x (gather_div = k)
+  const int32_t* gather_idx;  // row_src, or row_pair (token = row_pair / k)
+  int gather_div;
+  const void *w1, *w3, *w2;
+  void* h;                    // [P, f] bf16 scratch
+  void* o;                    // [P, d] bf16 out
+  const float* topk_w;        // NULL: un-weighted epilogue
+  const int32_t* row_pair;
+  const int32_t* expert_offsets;
+  const int32_t* mt_prefix;
+  int32_t* status;
+};
+cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st);
+int sm_count();
+
+}  // namespace tcmoe

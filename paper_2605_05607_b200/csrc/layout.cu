@@ -1,0 +1,316 @@
+// Dispatch layout, dispatch and combine (paper Sec. III-D: switch routing rule
+// group = expert / experts_per_group, AL tables built by a running counter, MV translation;
+// Sec. IV-B TID table; Sec. III-C un-weighted reduction in Combine).
+//
+// The hardware of the paper hands out layout rows in arrival order.  Here the order is fixed to
+// ascending token index so that the layout is a pure function of topk_idx: membership bitmasks
+// (one bit per (expert, token) and per (group, token)) are built with order-independent atomicOr,
+// an exclusive popcount scan along each mask row gives every token its rank, and a fill pass
+// turns ranks into the row tables.  No atomics touch the result arrays.
+#include "common.cuh"
+
+#include <cuda_bf16.h>
+
+namespace tcmoe {
+
+// ---- K2a: membership masks -------------------------------------------------------------------
+__global__ void __launch_bounds__(256) build_masks_kernel(const int32_t* __restrict__ topk_idx, uint32_t* emask,
+                                                          uint32_t* gmask, int T, int E, int k, int m, int W,
+                                                          int32_t* status) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;  // warp w covers tokens 32w .. 32w+31
+  const int lane = threadIdx.x & 31;
+  const int word = t >> 5;
+  const bool live = t < T;
+  for (int j = 0; j < k; ++j) {
+    int e = live ? __ldg(topk_idx + (size_t)t * k + j) : -1;
+    if (live && (e < 0 || e >= E)) {
+      report_error(status, DEV_INDEX_OUT_OF_RANGE, KID_MASKS, t, e);
+      e = -1;
+    }
+    // lanes that picked the same expert (group) fold their bits into one atomicOr
+    const unsigned same_e = __match_any_sync(0xFFFFFFFFu, e);
+    if (e >= 0 && lane == __ffs(same_e) - 1) atomicOr(&emask[(size_t)e * W + word], same_e);
+    const int g = (e >= 0) ? e / m : -1;
+    const unsigned same_g = __match_any_sync(0xFFFFFFFFu, g);
+    if (g >= 0 && lane == __ffs(same_g) - 1) atomicOr(&gmask[(size_t)g * W + word], same_g);
+  }
+}
+
+// ---- K2b: exclusive popcount prefix along every mask row; row totals -> counts ------------------
+__global__ void __launch_bounds__(256) scan_masks_kernel(const uint32_t* __restrict__ emask,
+                                                         const uint32_t* __restrict__ gmask, int32_t* eprefix,
+                                                         int32_t* gprefix, int32_t* expert_counts,
+                                                         int32_t* group_counts, int E, int W) {
+  __shared__ int warp_sum[8];
+  __shared__ int running_s;
+  const int row = blockIdx.x;
+  const uint32_t* mask = (row < E) ? emask + (size_t)row * W : gmask + (size_t)(row - E) * W;
+  int32_t* prefix = (row < E) ? eprefix + (size_t)row * W : gprefix + (size_t)(row - E) * W;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  if (threadIdx.x == 0) running_s = 0;
+  __syncthreads();
+  for (int base = 0; base < W; base += 256) {
+    const int i = base + threadIdx.x;
+    const int c = (i < W) ? __popc(mask[i]) : 0;
+    int incl = c;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int n = __shfl_up_sync(0xFFFFFFFFu, incl, off);
+      if (lane >= off) incl += n;
+    }
+    if (lane == 31) warp_sum[wid] = incl;
+    __syncthreads();
+    int warp_base = 0;
+    for (int w = 0; w < wid; ++w) warp_base += warp_sum[w];
+    const int running = running_s;
+    if (i < W) prefix[i] = running + warp_base + incl - c;
+    __syncthreads();
+    if (threadIdx.x == 255) running_s = running + warp_base + incl;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    if (row < E) expert_counts[row] = running_s;
+    else group_counts[row - E] = running_s;
+  }
+}
+
+// ---- K2c: offsets (exclusive scans over experts / groups) and the 128-row tile prefix -----------
+__global__ void __launch_bounds__(1024) offsets_kernel(const int32_t* __restrict__ expert_counts,
+                                                       const int32_t* __restrict__ group_counts,
+                                                       int32_t* expert_offsets, int32_t* group_offsets,
+                                                       int32_t* mt_prefix, int E, int G) {
+  __shared__ int buf[3][1024];
+  const int i = threadIdx.x;
+  const int ce = (i < E) ? expert_counts[i] : 0;
+  const int cg = (i < G) ? group_counts[i] : 0;
+  buf[0][i] = ce;
+  buf[1][i] = cg;
+  buf[2][i] = (ce + 127) >> 7;
+  __syncthreads();
+  for (int off = 1; off < 1024; off <<= 1) {  // Hillis-Steele inclusive scan, three lanes at once
+    int a = 0, b = 0, c = 0;
+    if (i >= off) { a = buf[0][i - off]; b = buf[1][i - off]; c = buf[2][i - off]; }
+    __syncthreads();
+    buf[0][i] += a; buf[1][i] += b; buf[2][i] += c;
+    __syncthreads();
+  }
+  if (i < E) { expert_offsets[i + 1] = buf[0][i]; mt_prefix[i + 1] = buf[2][i]; }
+  if (i < G) group_offsets[i + 1] = buf[1][i];
+  if (i == 0) { expert_offsets[0] = 0; group_offsets[0] = 0; mt_prefix[0] = 0; }
+}
+
+// ---- K2d: ranks -> row tables ----------------------------------------------------------------
+__global__ void __launch_bounds__(256) fill_layout_kernel(const int32_t* __restrict__ topk_idx, Layout L,
+                                                          LayoutScratch sc, int T, int E, int k, int G, int m) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
+  const int word = t >> 5;
+  const uint32_t below = (1u << (t & 31)) - 1u;
+  for (int g = 0; g < G; ++g) {
+    const uint32_t bits = sc.gmask[(size_t)g * sc.W + word];
+    int a = -1;
+    if (bits >> (t & 31) & 1u) {
+      a = sc.gprefix[(size_t)g * sc.W + word] + __popc(bits & below);
+      L.disp_token[L.group_offsets[g] + a] = t;  // TID table entry of the allocated row
+    }
+    L.al[(size_t)g * T + t] = a;
+  }
+  for (int j = 0; j < k; ++j) {
+    const int e = __ldg(topk_idx + (size_t)t * k + j);
+    if (e < 0 || e >= E) continue;  // already reported by build_masks_kernel
+    const int rank = sc.eprefix[(size_t)e * sc.W + word] + __popc(sc.emask[(size_t)e * sc.W + word] & below);
+    const int r = L.expert_offsets[e] + rank;
+    const int g = e / m;
+    const uint32_t gbits = sc.gmask[(size_t)g * sc.W + word];
+    const int a = sc.gprefix[(size_t)g * sc.W + word] + __popc(gbits & below);
+    L.pair_row[(size_t)t * k + j] = r;
+    L.row_pair[r] = t * k + j;
+    L.row_src[r] = L.group_offsets[g] + a;
+  }
+}
+
+// exclusive prefix of 128-row tiles per expert, from the counts alone
+__global__ void __launch_bounds__(1024) mt_prefix_kernel(const int32_t* __restrict__ expert_counts,
+                                                         int32_t* mt_prefix, int E) {
+  __shared__ int buf[1024];
+  const int i = threadIdx.x;
+  buf[i] = (i < E) ? (expert_counts[i] + 127) >> 7 : 0;
+  __syncthreads();
+  for (int off = 1; off < 1024; off <<= 1) {
+    const int a = (i >= off) ? buf[i - off] : 0;
+    __syncthreads();
+    buf[i] += a;
+    __syncthreads();
+  }
+  if (i < E) mt_prefix[i + 1] = buf[i];
+  if (i == 0) mt_prefix[0] = 0;
+}
+
+cudaError_t launch_mt_prefix(const Shape& s, const int32_t* expert_counts, int32_t* mt_prefix, cudaStream_t st) {
+  mt_prefix_kernel<<<1, 1024, 0, st>>>(expert_counts, mt_prefix, s.E);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_layout(const Shape& s, const int32_t* topk_idx, const Layout& L, const LayoutScratch& sc,
+                          int32_t* status, cudaStream_t st) {
+  const int m = s.E / s.G;
+  cudaError_t err;
+  if ((err = cudaMemsetAsync(sc.emask, 0, sizeof(uint32_t) * (size_t)(s.E + s.G) * sc.W, st)) != cudaSuccess)
+    return err;  // emask and gmask are adjacent
+  const int tb = (s.T + 255) / 256;
+  if (s.T > 0) build_masks_kernel<<<tb, 256, 0, st>>>(topk_idx, sc.emask, sc.gmask, s.T, s.E, s.k, m, sc.W, status);
+  scan_masks_kernel<<<s.E + s.G, 256, 0, st>>>(sc.emask, sc.gmask, sc.eprefix, sc.gprefix, L.expert_counts,
+                                                L.group_counts, s.E, sc.W);
+  offsets_kernel<<<1, 1024, 0, st>>>(L.expert_counts, L.group_counts, L.expert_offsets, L.group_offsets,
+                                     sc.mt_prefix, s.E, s.G);
+  if (s.T > 0) fill_layout_kernel<<<tb, 256, 0, st>>>(topk_idx, L, sc, s.T, s.E, s.k, s.G, m);
+  return cudaGetLastError();
+}
+
+// ---- K3: dispatch ------------------------------------------------------------------------------
+// Token-centric: a warp reads row x[t] once (16-byte vectors) and writes one copy per distinct
+// group the token touches - the single-HBM image of "send once, the switch replicates per port".
+__global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__ x, uint4* __restrict__ xg,
+                                                       const int32_t* __restrict__ al,
+                                                       const int32_t* __restrict__ group_offsets, int T, int G,
+                                                       int vec_per_row) {
+  const int lane = threadIdx.x & 31;
+  const int wpb = blockDim.x >> 5;
+  for (int t = blockIdx.x * wpb + (threadIdx.x >> 5); t < T; t += gridDim.x * wpb) {
+    const uint4* src = x + (size_t)t * vec_per_row;
+    for (int g0 = 0; g0 < G; g0 += 32) {
+      const int g = g0 + lane;
+      int dst_row = -1;
+      if (g < G) {
+        const int a = __ldg(al + (size_t)g * T + t);
+        if (a >= 0) dst_row = __ldg(group_offsets + g) + a;
+      }
+      unsigned live = __ballot_sync(0xFFFFFFFFu, dst_row >= 0);
+      if (!live) continue;
+      for (int v0 = 0; v0 < vec_per_row; v0 += 128) {
+        uint4 buf[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const int v = v0 + q * 32 + lane;
+          if (v < vec_per_row) buf[q] = __ldcs(src + v);
+        }
+        for (unsigned rem = live; rem; rem &= rem - 1) {
+          const int row = __shfl_sync(0xFFFFFFFFu, dst_row, __ffs(rem) - 1);
+          uint4* dst = xg + (size_t)row * vec_per_row;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            const int v = v0 + q * 32 + lane;
+            if (v < vec_per_row) __stcs(dst + v, buf[q]);
+          }
+        }
+      }
+    }
+  }
+}
+
+cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void* xg, cudaStream_t st) {
+  if (s.T == 0) return cudaSuccess;
+  int blocks = (s.T + 7) / 8;
+  const int cap = sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  dispatch_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(xg), L.al,
+                                          L.group_offsets, s.T, s.G, s.d / 8);
+  return cudaGetLastError();
+}
+
+// ---- K5: combine -----------------------------------------------------------------------------
+// One warp per token.  The k slots are visited group by group (ascending group, ascending slot
+// inside a group): the rows of one group are summed first (the pre-reduction that the switch
+// performs per output port), then the group partial joins the token's total; fp32 throughout.
+__device__ __forceinline__ void add_bf16x8(float (&acc)[8], const uint4& raw, float w) {
+  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float2 f = __bfloat1622float2(p[q]);
+    acc[2 * q] = fmaf(w, f.x, acc[2 * q]);
+    acc[2 * q + 1] = fmaf(w, f.y, acc[2 * q + 1]);
+  }
+}
+__device__ __forceinline__ uint4 pack_bf16x8(const float (&v)[8]) {
+  uint4 out;
+  __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&out);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) p[q] = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
+  return out;
+}
+
+__global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ o, uint4* __restrict__ y,
+                                                      uint4* __restrict__ pg, const int32_t* __restrict__ topk_idx,
+                                                      const float* __restrict__ topk_w,
+                                                      const int32_t* __restrict__ pair_row,
+                                                      const int32_t* __restrict__ al,
+                                                      const int32_t* __restrict__ group_offsets, int T, int k, int m,
+                                                      int vec_per_row, int weighted) {
+  __shared__ int s_row[8][32];   // per warp: expert-sorted row of the slot at sorted position p
+  __shared__ int s_dst[8][32];   // dispatched row (t, g) of that slot's group
+  __shared__ float s_w[8][32];
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const int wpb = blockDim.x >> 5;
+  for (int t = blockIdx.x * wpb + wid; t < T; t += gridDim.x * wpb) {
+    // lane j < k owns slot j; order slots by (group, slot)
+    int my_g = 0x7FFFFFFF, my_row = 0, my_dst = 0;
+    float my_w = 1.f;
+    if (lane < k) {
+      my_g = __ldg(topk_idx + (size_t)t * k + lane) / m;
+      my_row = __ldg(pair_row + (size_t)t * k + lane);
+      my_dst = __ldg(group_offsets + my_g) + __ldg(al + (size_t)my_g * T + t);
+      if (weighted) my_w = __ldg(topk_w + (size_t)t * k + lane);
+    }
+    int my_pos = 0;  // number of slots that come before mine
+    for (int j = 0; j < k; ++j) {
+      const int gj = __shfl_sync(0xFFFFFFFFu, my_g, j);
+      if (gj < my_g || (gj == my_g && j < lane)) ++my_pos;
+    }
+    __syncwarp();
+    if (lane < k) { s_row[wid][my_pos] = my_row; s_dst[wid][my_pos] = my_dst; s_w[wid][my_pos] = my_w; }
+    __syncwarp();
+    for (int v = lane; v < vec_per_row; v += 32) {
+      float total[8], part[8];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { total[q] = 0.f; part[q] = 0.f; }
+      int prev_dst = -1;
+      for (int s0 = 0; s0 < k; s0 += 8) {
+        uint4 buf[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q)   // all loads of the batch are in flight before the first use
+          if (s0 + q < k) buf[q] = __ldcs(o + (size_t)s_row[wid][s0 + q] * vec_per_row + v);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          if (s0 + q < k) {
+            const int dst = s_dst[wid][s0 + q];
+            if (dst != prev_dst && prev_dst >= 0) {   // a group is complete: emit its partial sum
+              if (pg != nullptr) pg[(size_t)prev_dst * vec_per_row + v] = pack_bf16x8(part);
+#pragma unroll
+              for (int c = 0; c < 8; ++c) { total[c] += part[c]; part[c] = 0.f; }
+            }
+            prev_dst = dst;
+            add_bf16x8(part, buf[q], s_w[wid][s0 + q]);
+          }
+        }
+      }
+      if (pg != nullptr) pg[(size_t)prev_dst * vec_per_row + v] = pack_bf16x8(part);
+#pragma unroll
+      for (int c = 0; c < 8; ++c) total[c] += part[c];
+      y[(size_t)t * vec_per_row + v] = pack_bf16x8(total);
+    }
+  }
+}
+
+cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
+                           const float* topk_w, void* pg, void* y, cudaStream_t st) {
+  if (s.T == 0) return cudaSuccess;
+  int blocks = (s.T + 7) / 8;
+  const int cap = sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  combine_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(o), static_cast<uint4*>(y),
+                                         static_cast<uint4*>(pg), topk_idx, topk_w, L.pair_row, L.al, L.group_offsets,
+                                         s.T, s.k, s.E / s.G, s.d / 8, (s.flags & 1) ? 1 : 0);
+  return cudaGetLastError();
+}
+
+}  // namespace tcmoe

@@ -1,0 +1,174 @@
+"""GPU parity tests: every stage of the path, called through the C ABI, against
+the CPU oracle on the same seeded inputs.  Integers bit-exact; outputs within
+max|gpu-ref| <= 2e-2 max|ref| and sum|gpu-ref|/sum|ref| <= 5e-3; logits 1e-4."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as O
+from paper_2605_05607_b200 import binding as B
+from paper_2605_05607_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+C1 = synth.CONFIGS["C1"]
+SMALL = [
+    C1,
+    C1.with_(name="C1-sigmoid-wcombine", score_fn=1),
+    # ragged everything: T not a multiple of 32/128, d and f with K/N tails, empty experts likely
+    synth.MoEConfig("ragged", T=333, d=200, f=328, E=12, k=3, G=4, bias="zipf", zipf_s=1.5, seed=2),
+    synth.MoEConfig("k1", T=150, d=128, f=192, E=4, k=1, G=2, seed=3),
+    synth.MoEConfig("kE-G1", T=70, d=64, f=64, E=4, k=4, G=1, seed=4),
+    synth.MoEConfig("G=E-local", T=200, d=256, f=128, E=16, k=4, G=16, bias="locality", boost=2.0, seed=5),
+    synth.MoEConfig("one-expert", T=300, d=192, f=448, E=1, k=1, G=1, seed=6),
+    synth.MoEConfig("gptoss-ish", T=512, d=2880 // 5, f=2880 // 5, E=32, k=4, G=8, bias="zipf", zipf_s=1.1, seed=7),
+]
+
+
+def staged(cfg, flags=0):
+    run = H.Run(cfg, flags)
+    run.route()
+    idx_ref, w_ref = H.check_route(run)
+    run.dispatch()
+    lay = H.check_layout(run, idx_ref)
+    n = lay["n_disp"]
+    xb = H.bf16_host(run.t["x"])
+    xg_ref = O.dispatch(xb, lay)
+    assert np.array_equal(H.bf16_host(run.xg)[:n], xg_ref), "dispatch is not a byte copy"
+    run.ffn()
+    w_gpu = run.host_w()
+    in_combine = bool(flags & B.MOE_FLAG_WEIGHT_IN_COMBINE)
+    o_ref = O.expert_ffn(xg_ref, lay, None if in_combine else w_gpu, H.bf16_host(run.t["w1"]),
+                         H.bf16_host(run.t["w3"]), H.bf16_host(run.t["w2"]))
+    o_gpu = O.bf16_to_f64(H.bf16_host(run.o)[: cfg.P])
+    H.assert_close_out(o_gpu, o_ref, "expert_ffn o")
+    pg = torch.zeros(max(n, 1), cfg.d, dtype=torch.bfloat16, device="cuda")
+    run.combine(pg)
+    # combine is checked against the oracle's combine of the GPU's own o (isolates this stage)
+    pg_n, pg_ref, y_ref = O.combine(o_gpu, lay, idx_ref, w_gpu if in_combine else None, cfg.E, cfg.G)
+    y_gpu = O.bf16_to_f64(H.bf16_host(run.y)[: cfg.T])
+    tol = 2.0 ** -8 * np.abs(y_ref) + 1e-30 + 2.0 ** -22 * np.abs(y_ref).max()
+    assert np.all(np.abs(y_gpu - y_ref) <= tol), "combine y"
+    pg_gpu = O.bf16_to_f64(H.bf16_host(pg)[:n])
+    tol = 2.0 ** -8 * np.abs(pg_ref) + 1e-30 + 2.0 ** -22 * max(np.abs(pg_ref).max(), 1e-30)
+    assert np.array_equal(pg_n, np.arange(n)) and np.all(np.abs(pg_gpu - pg_ref) <= tol), "combine pg"
+    # and the whole staged path against the dense definition
+    _, _, _, y_def = O.layer(xb, run.host_logits(), run.host_bias(), H.bf16_host(run.t["w1"]),
+                             H.bf16_host(run.t["w3"]), H.bf16_host(run.t["w2"]), cfg.k, cfg.score_fn)
+    H.assert_close_out(y_gpu, y_def, "staged y")
+    st = run.status()
+    assert st[0] == 0 and st[4] == 0, f"device status {st}"
+    return run, y_gpu, y_def
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
+def test_staged_path_matches_oracle(cfg):
+    flags = B.MOE_FLAG_WEIGHT_IN_COMBINE if "wcombine" in cfg.name else 0
+    staged(cfg, flags)
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
+def test_fused_layer_matches_oracle_and_staged(cfg):
+    run, y_staged, y_def = staged(cfg)
+    y2 = torch.zeros_like(run.y)
+    logits = torch.zeros_like(run.logits)
+    idx = torch.zeros_like(run.idx)
+    w = torch.zeros_like(run.w)
+    lay2 = B.alloc_layout(run.shape)
+    run.layer(y=y2, logits=logits, topk_idx=idx, topk_w=w, layout=lay2)
+    assert torch.equal(idx, run.idx) and torch.equal(logits, run.logits) and torch.equal(w, run.w)
+    for name in ("expert_offsets", "group_offsets", "pair_row", "row_pair", "row_src", "al"):
+        assert torch.equal(getattr(lay2, name), getattr(run.lay, name)), name
+    y_fused = O.bf16_to_f64(H.bf16_host(y2)[: cfg.T])
+    H.assert_close_out(y_fused, y_def, "fused y")
+    # gathering from x instead of the dispatched copy feeds the GEMM the same bytes
+    assert np.array_equal(y_fused, y_staged)
+    # optional outputs left NULL: same y
+    y3 = torch.zeros_like(run.y)
+    run.layer(y=y3)
+    assert torch.equal(y3, y2)
+    assert run.status()[0] == 0
+
+
+def test_topk_ties_lowest_index_wins():
+    # logits quantised to a handful of values: ties everywhere, incl. at the k / k+1 border
+    cfg = synth.MoEConfig("ties", T=777, d=64, f=64, E=40, k=6, G=4)
+    run = H.Run(cfg, inputs=synth.make_routing_inputs(cfg, "cuda") | {"w1": None, "w3": None, "w2": None})
+    g = torch.Generator(device="cuda").manual_seed(11)
+    vals = torch.tensor([-1.0, -0.0, 0.0, 0.5, 0.5, 2.0], device="cuda")
+    logits = vals[torch.randint(0, 6, (cfg.T, cfg.E), generator=g, device="cuda")].contiguous()
+    run.logits = logits.reshape(-1).clone()
+    for score_fn in (0, 1):
+        shape = B.make_shape(cfg.with_(score_fn=score_fn))
+        B.moe_route(shape, None, None, None, run.logits, run.idx, run.w, run.ws)
+        idx_ref, w_ref = O.route(logits.cpu().numpy(), None, cfg.k, score_fn)
+        assert np.array_equal(run.host_idx(), idx_ref)
+        assert np.abs(run.host_w() - w_ref).max() <= H.WEIGHT_ABS
+    # all-equal keys -> experts 0..k-1, weights 1/k
+    run.logits.fill_(0.25)
+    B.moe_route(run.shape, None, None, None, run.logits, run.idx, run.w, run.ws)
+    assert np.array_equal(run.host_idx(), np.tile(np.arange(cfg.k, dtype=np.int32), (cfg.T, 1)))
+    assert np.allclose(run.host_w(), 1.0 / cfg.k, atol=1e-7)
+    assert run.status()[5] == 0
+
+
+def test_bias_forms_and_nonfinite_warning():
+    cfg = synth.MoEConfig("bias", T=100, d=64, f=64, E=64, k=4, G=8, bias="locality", boost=2.0, seed=9)
+    run = H.Run(cfg, inputs=synth.make_routing_inputs(cfg, "cuda") | {"w1": None, "w3": None, "w2": None})
+    run.route()
+    H.check_route(run)                                   # [T, E] bias
+    zcfg = cfg.with_(bias="zipf", zipf_s=1.2)
+    run2 = H.Run(zcfg, inputs=synth.make_routing_inputs(zcfg, "cuda") | {"w1": None, "w3": None, "w2": None})
+    run2.route()
+    H.check_route(run2)                                  # [E] bias
+    assert run2.status()[5] == 0
+    run2.logits[5] = float("inf")
+    B.moe_route(run2.shape, None, None, run2.t["bias"], run2.logits, run2.idx, run2.w, run2.ws)
+    assert run2.status()[5] & B.MOE_WARN_NONFINITE_LOGIT
+
+
+def test_combine_identity_experts_and_linearity():
+    # "identity experts": feed o[r] := xg[row_src[r]]; weights sum to 1, so combine returns x
+    for k in (1, 2, 4):
+        cfg = synth.MoEConfig(f"ident{k}", T=260, d=520, f=64, E=8, k=k, G=4, seed=k)
+        run = H.Run(cfg, B.MOE_FLAG_WEIGHT_IN_COMBINE,
+                    inputs=synth.make_routing_inputs(cfg, "cuda") | {"w1": None, "w3": None, "w2": None})
+        run.route()
+        run.dispatch()
+        run.o = run.xg[run.lay.row_src[: cfg.P].long()].contiguous()
+        run.combine()
+        x = O.bf16_to_f64(H.bf16_host(run.t["x"]))
+        y = O.bf16_to_f64(H.bf16_host(run.y)[: cfg.T])
+        if k == 1:
+            assert np.array_equal(y, x)                  # pure un-permute, bit-exact
+        else:
+            assert np.all(np.abs(y - x) <= 2.0 ** -7 * np.abs(x) + 1e-30)
+        # linearity in a power of two is exact
+        y1 = run.y.clone()
+        run.o = (run.o.float() * 4.0).to(torch.bfloat16)
+        run.combine()
+        assert torch.equal(run.y.float(), y1.float() * 4.0)
+
+
+def test_degenerate_and_error_paths():
+    cfg = synth.MoEConfig("empty", T=0, d=64, f=64, E=4, k=2, G=2)
+    run = H.Run(cfg, inputs={"x": torch.zeros(1, 64, dtype=torch.bfloat16, device="cuda"),
+                             "w_gate": torch.zeros(64, 4, device="cuda"), "bias": None,
+                             "w1": torch.zeros(4, 64, 64, dtype=torch.bfloat16, device="cuda"),
+                             "w3": torch.zeros(4, 64, 64, dtype=torch.bfloat16, device="cuda"),
+                             "w2": torch.zeros(4, 64, 64, dtype=torch.bfloat16, device="cuda")})
+    run.route(); run.dispatch(); run.ffn(); run.combine(); run.layer()
+    torch.cuda.synchronize()
+    assert run.status()[0] == 0
+    assert run.lay.expert_offsets[:5].tolist() == [0] * 5
+    # an out-of-range expert index is reported, not dereferenced
+    cfg = synth.MoEConfig("badidx", T=40, d=64, f=64, E=4, k=2, G=2)
+    run = H.Run(cfg, inputs=synth.make_routing_inputs(cfg, "cuda") | {"w1": None, "w3": None, "w2": None})
+    run.route()
+    run.idx[7] = 99
+    run.dispatch()
+    st = run.status()
+    assert st[0] == B.MOE_DEV_INDEX_OUT_OF_RANGE and st[3] == 99
+    B.moe_status_reset(run.ws)
+    assert run.status()[0] == 0
