@@ -1,0 +1,304 @@
+"""Benchmark of the fused MoE layer (gate -> layout -> expert FFN -> combine) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C2] [--impl reference]
+
+One step = one pass of the whole hot path (moe_layer) over one batch of synthetic tokens.
+N > 1 (launched by torchrun): every rank runs an independent replica on its own tokens (weights
+replicated, tokens sharded, no data-path collective) - weak scaling.  Rank 0 prints ONE JSON line.
+`--impl reference` times the CPU oracle on a bounded token sample instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+import torch  # noqa: E402
+
+from paper_2605_05607_b200 import synth  # noqa: E402
+
+METRIC = "fused MoE layer tokens/sec"
+UNIT = "tokens/s"
+KERNELS_PER_STEP = 9  # gate, topk, masks, scan, offsets, fill, gemm1, gemm2, combine
+
+# DRAM bytes (read + write) of one GEMM-1 launch from ncu captures summarised under profiles/;
+# None until a capture of that workload exists.
+GEMM1_DRAM_TRAFFIC = {}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks / throttle reasons of one GPU while the benchmark runs."""
+    Q = ("uuid,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.uuid = uuid
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            return
+        def pump():
+            for line in self.proc.stdout:
+                f = [c.strip() for c in line.split(",")]
+                if len(f) >= 9 and (self.uuid in f[0] or f[0] in self.uuid):
+                    self.rows.append((time.time(), f))
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        rows = [f for (ts, f) in self.rows if t0 <= ts <= t1]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm = sorted(float(f[1]) for f in rows)
+        reasons = set()
+        for f in rows:
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(rows[0][2]),
+                "power_w_max": max(float(f[3]) for f in rows), "reasons": sorted(reasons), "samples": len(rows)}
+
+
+def oracle_sample_run(cfg, t, sample: int):
+    """Time the CPU oracle (as it stands) on `sample` tokens of the workload; returns seconds."""
+    from oracle import moe_oracle as O
+    bits = synth.bf16_bits
+    xb = bits(t["x"])
+    w1, w3, w2 = bits(t["w1"]), bits(t["w3"]), bits(t["w2"])
+    wg = t["w_gate"].cpu().numpy()
+    bias = None if t["bias"] is None else t["bias"].cpu().numpy()
+    toks = synth.sample_tokens(cfg, sample)
+    t0 = time.perf_counter()
+    logits = O.gate_logits(xb[toks], wg)                     # gate of the sampled tokens
+    b = bias if bias is None or bias.ndim == 1 else bias[toks]
+    O.layer(xb[toks], logits, b, w1, w3, w2, cfg.k, cfg.score_fn)
+    return time.perf_counter() - t0, len(toks)
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    t = synth.make_inputs(cfg, "cpu")
+    sample = args.ref_sample
+    if sample <= 0:
+        # size the per-step sample so that the whole run stays within ~200 s: one token is timed
+        # first; n tokens never cost more than n times that (weight decoding is shared)
+        dt1, _ = oracle_sample_run(cfg, t, 1)
+        sample = int(max(1, min(64, 200.0 / (args.steps + args.warmup) / dt1)))
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt, n = oracle_sample_run(cfg, t, sample)
+        if i >= args.warmup:
+            times.append(dt)
+    per_step = float(np.mean(times))
+    value = n / per_step
+    cores = blas_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(cfg, args.gpus),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{n} of {cfg.T} tokens per step (gate + top-k + expert FFN + combine)"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, n_gpus):
+    return {"workload": f"{cfg.name}: T={cfg.T} d={cfg.d} f={cfg.f} E={cfg.E} top-{cfg.k} G={cfg.G} per GPU",
+            "T": cfg.T, "d": cfg.d, "f": cfg.f, "E": cfg.E, "k": cfg.k, "G": cfg.G,
+            "score_fn": "softmax" if cfg.score_fn == 0 else "sigmoid", "router_bias": cfg.bias,
+            "parallelism": f"replicas x{n_gpus} (tokens sharded, weights replicated, no collective)",
+            "l2": "inputs larger than L2: expert weights %.2f GB streamed every step" %
+                  (6.0 * cfg.E * cfg.d * cfg.f / 1e9)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="C2", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--impl", default="tcmoe", choices=["tcmoe", "reference"])
+    ap.add_argument("--ref-sample", type=int, default=0,
+                    help="tokens per step of the reference arm (0: sized from a one-token calibration)")
+    ap.add_argument("--cpu-sample", type=int, default=64, help="tokens of the cpu_baseline leg (0: skip)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "tcmoe" else args.warmup
+    cfg = synth.CONFIGS[args.config]
+
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    from paper_2605_05607_b200 import binding as B
+    B.lib()  # fail loudly if the CUDA library is missing
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # weights replicated (same seed on every rank), tokens differ per rank
+    t = synth.make_inputs(cfg, "cuda")
+    if rank > 0:
+        t["x"] = synth.make_routing_inputs(cfg.with_(seed=cfg.seed + 7919 * rank), "cuda")["x"]
+    shape = B.make_shape(cfg)
+    ws = B.alloc_workspace(shape)
+    y = torch.zeros(cfg.T, cfg.d, dtype=torch.bfloat16, device="cuda")
+
+    def step():
+        B.moe_layer(shape, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws)
+
+    sampler = None
+    if rank == 0:
+        sampler = ClockSampler(str(torch.cuda.get_device_properties(local).uuid))
+        sampler.start()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region: K steps, CUDA events on the launching stream, GEMM-1 bracketed per launch
+    B.moe_profile_enable(B.KERNEL_IDS["gemm1"])
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    wall0 = time.time()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    wall1 = time.time()
+    elapsed_ms = ev0.elapsed_time(ev1)
+    g1_ms, g1_launches = B.moe_profile_read()
+    B.moe_profile_enable(0)
+    if dist is not None:
+        tmax = torch.tensor([elapsed_ms], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tmax.item())
+    status = B.moe_status(ws)
+    assert status[0] == 0, f"device status {status}"
+
+    # ---- end to end through the host-buffer entry point: pinned x in, y out, every step
+    x_host = t["x"].cpu().pin_memory()
+    y_host = torch.empty_like(x_host).pin_memory()
+    x_dev = torch.empty_like(t["x"])
+    for _ in range(3):
+        B.moe_layer_host(shape, x_host, x_dev, t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, y_host, ws)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        B.moe_layer_host(shape, x_host, x_dev, t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, y_host, ws)
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        tmax = torch.tensor([e2e_ms], device="cuda")
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tmax.item())
+
+    clocks = None
+    if sampler is not None:
+        clocks = sampler.summary(wall0, wall1)
+        if clocks["samples"] < 3:  # timed region too short for the 100 ms sampler: keep the same load running
+            p0 = time.time()
+            while time.time() - p0 < 1.5:
+                for _ in range(10):
+                    step()
+                torch.cuda.synchronize()
+            clocks = sampler.summary(p0, time.time())
+            clocks["window"] = "same load repeated for 1.5 s after the timed region"
+        sampler.stop()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    tokens = cfg.T * world * args.steps
+    value = tokens / (elapsed_ms * 1e-3)
+    flops_g1 = 4.0 * cfg.P * cfg.d * cfg.f                      # GEMM-1: x W1 and x W3
+    g1_avg_s = (g1_ms / max(g1_launches, 1)) * 1e-3
+    achieved = flops_g1 / g1_avg_s / 1e12 if g1_launches else None
+    peak = pk["bf16_tflops_sustained"]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic", "config": workload_config(cfg, world),
+        "clocks": clocks,
+        "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.T * cfg.d * 2,
+                "d2h_bytes_per_step": cfg.T * cfg.d * 2},
+        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "roofline": {"kernel": "ffn_gemm_kernel<0> (GEMM-1 + SwiGLU, tcgen05)", "bound": "tensor",
+                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": (achieved / peak) if achieved else None,
+                     "peak_source": f"{pk['source']} bf16 sustained (kernel timed inside a long step)",
+                     "flops_per_launch": flops_g1, "avg_launch_ms": g1_avg_s * 1e3, "launches": g1_launches,
+                     "traffic": GEMM1_DRAM_TRAFFIC.get(cfg.name)},
+        "ffn_tflops_layer": 6.0 * cfg.P * cfg.d * cfg.f * args.steps / (elapsed_ms * 1e-3) / 1e12,
+    }
+    if world == 1 and args.cpu_sample > 0:
+        dt, n = oracle_sample_run(cfg, t, args.cpu_sample)
+        line["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                                "sample": f"{n} of {cfg.T} tokens, {dt:.1f} s (gate + top-k + expert FFN + combine)"}
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

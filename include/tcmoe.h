@@ -163,6 +163,19 @@ int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, co
  * by moe_layer, out[3] expert m-tile prefix [E+1] int32. */
 int moe_workspace_layout(const moe_shape_t* shape, size_t out[4]);
 
+/* Kernel ids for moe_profile_enable (also the `where` slot of moe_status). */
+enum { MOE_KERNEL_TOPK = 1, MOE_KERNEL_MASKS = 2, MOE_KERNEL_FILL = 3, MOE_KERNEL_DISPATCH = 4,
+       MOE_KERNEL_GEMM1 = 5, MOE_KERNEL_GEMM2 = 6, MOE_KERNEL_COMBINE = 7, MOE_KERNEL_GATE = 8 };
+
+/* Per-kernel timing hook for benchmarks (host-side state, one per process; not part of the
+ * method).  After moe_profile_enable(id) every launch of that kernel by any entry point is
+ * bracketed by a pair of CUDA events on the launching stream (up to 4096 launches; later ones
+ * are not recorded).  moe_profile_read waits for the recorded events, returns the summed
+ * device time in milliseconds and the number of launches, and clears the record.
+ * moe_profile_enable(0) switches the hook off. */
+int moe_profile_enable(int kernel_id);
+int moe_profile_read(float* total_ms, int32_t* launches);
+
 #ifdef __cplusplus
 }
 #endif

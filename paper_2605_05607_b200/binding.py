@@ -31,7 +31,8 @@ MOE_WARN_NONFINITE_LOGIT = 1
 MOE_FLAG_WEIGHT_IN_COMBINE = 1
 
 EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "moe_status", "moe_strerror",
-           "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host")
+           "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",
+           "moe_profile_enable", "moe_profile_read")
 
 
 class MoEShape(ctypes.Structure):
@@ -75,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.moe_combine.argtypes = [shp, vp, lay, vp, vp, vp, vp, vp, sz, vp]
         L.moe_layer.argtypes = [shp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, lay, vp, sz, vp]
         L.moe_layer_host.argtypes = [shp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.moe_profile_enable.argtypes = [ctypes.c_int]
+        L.moe_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
         for name in EXPORTS:
             if name != "moe_strerror":
                 getattr(L, name).restype = ctypes.c_int
@@ -199,3 +202,17 @@ def moe_layer_host(shape, x_host, x_dev, w_gate, logit_bias, w1, w3, w2, y_dev, 
     _check("moe_layer_host", lib().moe_layer_host(ctypes.byref(shape), _ptr(x_host), _ptr(x_dev), _ptr(w_gate),
                                                   _ptr(logit_bias), stride, _ptr(w1), _ptr(w3), _ptr(w2),
                                                   _ptr(y_dev), _ptr(y_host), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+KERNEL_IDS = {"topk": 1, "masks": 2, "fill": 3, "dispatch": 4, "gemm1": 5, "gemm2": 6, "combine": 7, "gate": 8}
+
+
+def moe_profile_enable(kernel_id: int) -> None:
+    _check("moe_profile_enable", lib().moe_profile_enable(kernel_id))
+
+
+def moe_profile_read():
+    """(total device milliseconds, launches) of the profiled kernel since the last read."""
+    ms, n = ctypes.c_float(0), ctypes.c_int32(0)
+    _check("moe_profile_read", lib().moe_profile_read(ctypes.byref(ms), ctypes.byref(n)))
+    return ms.value, n.value

@@ -127,9 +127,56 @@ bool have_device() {
 }  // namespace
 }  // namespace tcmoe
 
+namespace tcmoe {
+namespace {
+constexpr int PROFILE_CAP = 4096;
+int g_profile_id = 0;
+int g_profile_n = 0;
+cudaEvent_t g_ev0[PROFILE_CAP], g_ev1[PROFILE_CAP];
+int g_events_made = 0;
+}  // namespace
+
+ProfileScope::ProfileScope(int kernel_id, cudaStream_t s) : slot(-1), st(s) {
+  if (g_profile_id == 0 || kernel_id != g_profile_id || g_profile_n >= PROFILE_CAP) return;
+  while (g_events_made <= g_profile_n) {
+    if (cudaEventCreate(&g_ev0[g_events_made]) != cudaSuccess || cudaEventCreate(&g_ev1[g_events_made]) != cudaSuccess)
+      return;
+    ++g_events_made;
+  }
+  slot = g_profile_n++;
+  cudaEventRecord(g_ev0[slot], st);
+}
+ProfileScope::~ProfileScope() {
+  if (slot >= 0) cudaEventRecord(g_ev1[slot], st);
+}
+}  // namespace tcmoe
+
 using namespace tcmoe;
 
 extern "C" {
+
+int moe_profile_enable(int kernel_id) {
+  if (kernel_id < 0 || kernel_id > 8) return MOE_ERR_INVALID_ARG;
+  g_profile_id = kernel_id;
+  g_profile_n = 0;
+  return MOE_OK;
+}
+
+int moe_profile_read(float* total_ms, int32_t* launches) {
+  if (total_ms == nullptr || launches == nullptr) return MOE_ERR_INVALID_ARG;
+  float sum = 0.f;
+  for (int i = 0; i < g_profile_n; ++i) {
+    float ms = 0.f;
+    TCMOE_CUDA(cudaEventSynchronize(g_ev1[i]));
+    TCMOE_CUDA(cudaEventElapsedTime(&ms, g_ev0[i], g_ev1[i]));
+    sum += ms;
+  }
+  *total_ms = sum;
+  *launches = g_profile_n;
+  g_profile_n = 0;
+  return MOE_OK;
+}
+
 
 int moe_workspace_bytes(const moe_shape_t* shape, size_t* bytes) {
   int rc = check_shape(shape);

@@ -69,4 +69,12 @@ struct FfnArgs {
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st);
 int sm_count();
 
+// Optional event bracket around launches of one kernel id (see moe_profile_enable).
+struct ProfileScope {
+  ProfileScope(int kernel_id, cudaStream_t st);
+  ~ProfileScope();
+  int slot;
+  cudaStream_t st;
+};
+
 }  // namespace tcmoe

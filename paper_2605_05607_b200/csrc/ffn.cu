@@ -431,7 +431,10 @@ cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st)
   g1.N = s.f;
   g1.n_tiles = (s.f + 127) / 128;
   g1.status = a.status;
-  ffn_gemm_kernel<0><<<grid, 320, SMEM_BYTES, st>>>(m_w1, m_w3, m_h, g1);
+  {
+    ProfileScope prof(KID_GEMM1, st);
+    ffn_gemm_kernel<0><<<grid, 320, SMEM_BYTES, st>>>(m_w1, m_w3, m_h, g1);
+  }
   cudaError_t err = cudaGetLastError();
   if (err != cudaSuccess) return err;
 
@@ -447,7 +450,10 @@ cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st)
   g2.N = s.d;
   g2.n_tiles = (s.d + 255) / 256;
   g2.status = a.status;
-  ffn_gemm_kernel<1><<<grid, 192, SMEM_BYTES, st>>>(m_w2, m_w2, m_h, g2);
+  {
+    ProfileScope prof(KID_GEMM2, st);
+    ffn_gemm_kernel<1><<<grid, 192, SMEM_BYTES, st>>>(m_w2, m_w2, m_h, g2);
+  }
   return cudaGetLastError();
 }
 

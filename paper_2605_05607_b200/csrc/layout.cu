@@ -213,6 +213,7 @@ cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void
   int blocks = (s.T + 7) / 8;
   const int cap = sm_count() * 8;
   if (blocks > cap) blocks = cap;
+  ProfileScope prof(KID_DISPATCH, st);
   dispatch_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(xg), L.al,
                                           L.group_offsets, s.T, s.G, s.d / 8);
   return cudaGetLastError();
@@ -307,6 +308,7 @@ cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const
   int blocks = (s.T + 7) / 8;
   const int cap = sm_count() * 8;
   if (blocks > cap) blocks = cap;
+  ProfileScope prof(KID_COMBINE, st);
   combine_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(o), static_cast<uint4*>(y),
                                          static_cast<uint4*>(pg), topk_idx, topk_w, L.pair_row, L.al, L.group_offsets,
                                          s.T, s.k, s.E / s.G, s.d / 8, (s.flags & 1) ? 1 : 0);

@@ -90,6 +90,7 @@ __global__ void __launch_bounds__(256) gate_logits_kernel(const __nv_bfloat16* _
 template <int BN>
 static cudaError_t launch_gate_bn(const Shape& s, const void* x, const float* wg, float* logits, cudaStream_t st) {
   dim3 grid((s.T + GateCfg<BN>::BM - 1) / GateCfg<BN>::BM, (s.E + BN - 1) / BN);
+  ProfileScope prof(KID_GATE, st);
   gate_logits_kernel<BN><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), wg, logits, s.T, s.d, s.E);
   return cudaGetLastError();
 }
@@ -182,6 +183,7 @@ cudaError_t launch_topk(const Shape& s, const float* logits, const float* bias, 
   const int cap = sm_count() * 8;
   if (blocks > cap) blocks = cap;
   const int kpl = (s.E + 31) / 32;
+  ProfileScope prof(KID_TOPK, st);
 #define TCMOE_TOPK(KPL)                                                                                        \
   topk_kernel<KPL><<<blocks, warps * 32, 0, st>>>(logits, bias, (long long)bias_stride, topk_idx, topk_w, s.T, \
                                                   s.E, s.k, s.score_fn, status)

@@ -1,0 +1,129 @@
+"""CPU-side checks of the C-ABI boundary: the library loads, exports every symbol the header
+declares, sizes its workspace sensibly and rejects bad arguments before touching a device."""
+import ctypes
+import os
+import re
+
+import pytest
+import torch
+
+from paper_2605_05607_b200 import binding as B
+from paper_2605_05607_b200 import build, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return B.lib()
+
+
+def header_symbols():
+    text = open(os.path.join(ROOT, "include", "tcmoe.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(moe_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = header_symbols()
+    assert set(names) == set(B.EXPORTS), (names, B.EXPORTS)
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_strerror(lib):
+    assert B.strerror(0) == "ok"
+    assert "workspace" in B.strerror(B.MOE_ERR_WORKSPACE_TOO_SMALL)
+    assert "unknown" in B.strerror(12345)
+
+
+def test_workspace_bytes_and_layout(lib):
+    for name, cfg in synth.CONFIGS.items():
+        shape = B.make_shape(cfg)
+        n = B.moe_workspace_bytes(shape)
+        lay = B.moe_workspace_layout(shape)
+        P = cfg.T * cfg.k
+        assert n >= P * cfg.f * 2 + P * cfg.d * 2            # h and o live inside
+        assert lay["status"] == 0 and lay["h"] % 1024 == 0 and lay["o"] % 1024 == 0
+        assert lay["o"] - lay["h"] >= P * cfg.f * 2
+        assert n < 8e9, name
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(k=9), B.MOE_ERR_INVALID_ARG),            # k > E
+    (dict(G=3), B.MOE_ERR_INVALID_ARG),            # E % G != 0
+    (dict(T=-1), B.MOE_ERR_INVALID_ARG),
+    (dict(score_fn=2), B.MOE_ERR_INVALID_ARG),
+    (dict(d=100), B.MOE_ERR_UNSUPPORTED_SHAPE),    # d % 8 != 0
+    (dict(f=12), B.MOE_ERR_UNSUPPORTED_SHAPE),
+    (dict(E=2048, G=8, k=2), B.MOE_ERR_UNSUPPORTED_SHAPE),
+    (dict(E=64, k=33, G=8), B.MOE_ERR_UNSUPPORTED_SHAPE),
+    (dict(T=2 ** 30, k=2), B.MOE_ERR_UNSUPPORTED_SHAPE),
+])
+def test_bad_shapes_rejected(lib, kw, code):
+    cfg = synth.CONFIGS["C1"].with_(**kw)
+    with pytest.raises(B.MoEError) as ei:
+        B.moe_workspace_bytes(B.make_shape(cfg))
+    assert ei.value.code == code
+
+
+def test_bad_flags_rejected(lib):
+    with pytest.raises(B.MoEError) as ei:
+        B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=4))
+    assert ei.value.code == B.MOE_ERR_INVALID_ARG
+
+
+def test_argument_checks_happen_before_any_device_work(lib):
+    """Null / misaligned pointers and a short workspace are rejected on the host; with valid
+    arguments but no GPU the call reports MOE_ERR_CUDA instead of falling back to anything."""
+    cfg = synth.CONFIGS["C1"].with_(T=8)
+    shape = B.make_shape(cfg)
+    n = B.moe_workspace_bytes(shape)
+    ws = torch.zeros(n + 256, dtype=torch.uint8)
+    base = ws.data_ptr()
+    pad = (-base) % 128
+    ws_al = ws[pad: pad + n]
+    f32 = torch.zeros(cfg.T * cfg.E, dtype=torch.float32)
+    i32 = torch.zeros(cfg.T * cfg.k, dtype=torch.int32)
+    w = torch.zeros(cfg.T * cfg.k, dtype=torch.float32)
+
+    def rc(fn):
+        try:
+            fn()
+        except B.MoEError as e:
+            return e.code
+        return 0
+
+    # null outputs
+    assert rc(lambda: B.moe_route(shape, None, None, None, None, i32, w, ws_al)) == B.MOE_ERR_INVALID_ARG
+    # workspace too small
+    assert rc(lambda: B.moe_route(shape, None, None, None, f32, i32, w, ws_al[:1024])) == B.MOE_ERR_WORKSPACE_TOO_SMALL
+    # misaligned workspace
+    assert rc(lambda: B.moe_route(shape, None, None, None, f32, i32, w, ws[pad + 4: pad + 4 + n])) == B.MOE_ERR_MISALIGNED
+    # bias stride must be 0 or E
+    lib_rc = B.lib().moe_route(ctypes.byref(shape), None, None, f32.data_ptr(), 3, f32.data_ptr(), i32.data_ptr(),
+                               w.data_ptr(), ws_al.data_ptr(), n, None)
+    assert lib_rc == B.MOE_ERR_INVALID_ARG
+    # null layout
+    assert B.lib().moe_dispatch(ctypes.byref(shape), None, i32.data_ptr(), None, None, ws_al.data_ptr(), n,
+                                None) == B.MOE_ERR_INVALID_ARG
+    if not torch.cuda.is_available():
+        assert rc(lambda: B.moe_route(shape, None, None, None, f32, i32, w, ws_al)) == B.MOE_ERR_CUDA
+        assert rc(lambda: B.moe_status(ws_al)) == B.MOE_ERR_CUDA
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(B, "_lib_handle", None)
+    monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no CPU fallback"):
+        B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"]))
+
+
+def test_product_package_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2605_05607_b200")
+    pat = re.compile(r"^\s*(from|import)\s+oracle\b|oracle[/.]moe_oracle|#include\s+\".*oracle", re.M)
+    for dirpath, _, files in os.walk(pkg):
+        for fn in files:
+            if fn.endswith((".py", ".cu", ".cuh", ".h")):
+                assert not pat.search(open(os.path.join(dirpath, fn)).read()), fn

@@ -1,0 +1,80 @@
+"""Full-size parity: the five benchmark configurations through moe_layer (the launch configuration
+bench.py times).  Routing and layout are compared in full (bit-exact); expert outputs on sampled
+rows of sampled experts and the layer output on sampled tokens, one by one against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import moe_oracle as O
+from paper_2605_05607_b200 import binding as B
+from paper_2605_05607_b200 import synth
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+class Slabs:
+    """Expert weight matrices fetched from the device one expert at a time."""
+
+    def __init__(self, w):
+        self.w = w
+
+    def __getitem__(self, e):
+        return synth.bf16_bits(self.w[int(e)])
+
+
+@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5a", "C5b"])
+def test_fullsize_layer(name):
+    cfg = synth.CONFIGS[name]
+    run = H.Run(cfg)
+    lay_dev = B.alloc_layout(run.shape)
+    run.layer(logits=run.logits, topk_idx=run.idx, topk_w=run.w, layout=lay_dev)
+    torch.cuda.synchronize()
+    st = run.status()
+    assert st[0] == 0 and st[4] == 0, f"device status {st}"
+    run.lay = lay_dev
+    idx_ref, w_ref = H.check_route(run)               # logits 1e-4; idx bit-exact; weights 1e-6
+    lay = H.check_layout(run, idx_ref)                # counts / offsets / permutation bit-exact
+    P, T, k = cfg.P, cfg.T, cfg.k
+    assert lay["n_disp"] <= T * min(k, cfg.G)
+    if cfg.G == cfg.E:
+        assert lay["n_disp"] == P                     # one expert per group: nothing to de-duplicate
+
+    # expert outputs o (kept in the workspace by moe_layer): sampled rows of sampled experts
+    off = B.moe_workspace_layout(run.shape)
+    o_dev = run.ws[off["o"]: off["o"] + P * cfg.d * 2].view(torch.bfloat16).reshape(P, cfg.d)
+    counts = lay["expert_counts"]
+    live = np.nonzero(counts)[0]
+    rng = np.random.default_rng(1)
+    picks = {int(live[np.argmax(counts[live])]), int(live[np.argmin(counts[live])]), int(rng.choice(live))}
+    rows = []
+    for e in sorted(picks):
+        lo, hi = int(lay["expert_offsets"][e]), int(lay["expert_offsets"][e + 1])
+        take = np.unique(np.concatenate([np.arange(lo, min(lo + 8, hi)), np.arange(max(hi - 8, lo), hi),
+                                         rng.integers(lo, hi, size=8)]))
+        rows.append(take)
+    rows = np.unique(np.concatenate(rows))
+    xb = H.bf16_host(run.t["x"])
+    # the fused path feeds GEMM-1 from x; the oracle's dispatched copy holds the same bytes
+    xg = O.dispatch(xb, lay)
+    w_gpu = run.host_w()
+    o_ref = O.expert_ffn(xg, lay, w_gpu, Slabs(run.t["w1"]), Slabs(run.t["w3"]), Slabs(run.t["w2"]), rows=rows)
+    o_gpu = O.bf16_to_f64(H.bf16_host(o_dev[torch.from_numpy(rows).cuda()]))
+    H.assert_close_out(o_gpu, o_ref, f"{name} expert rows")
+
+    # combine on sampled tokens from the GPU's own o (all k rows of each token)
+    toks = synth.sample_tokens(cfg, 96)
+    need = np.unique(lay["pair_row"].reshape(T, k)[toks].reshape(-1))
+    o_need = O.bf16_to_f64(H.bf16_host(o_dev[torch.from_numpy(need).cuda()]))
+    _, _, y_ref = O.combine(o_need, lay, idx_ref, None, cfg.E, cfg.G, tokens=toks, o_rows=need)
+    y_gpu = O.bf16_to_f64(H.bf16_host(run.y[torch.from_numpy(toks).cuda()]))
+    tol = 2.0 ** -8 * np.abs(y_ref) + 2.0 ** -22 * np.abs(y_ref).max() + 1e-30
+    assert np.all(np.abs(y_gpu - y_ref) <= tol), f"{name} combine"
+
+    # whole layer against the dense definition on a few tokens
+    few = synth.sample_tokens(cfg, 96)[:: 96 // 4][:4]
+    b = run.host_bias()
+    _, _, _, y_def = O.layer(xb, run.host_logits(), b, Slabs(run.t["w1"]), Slabs(run.t["w3"]), Slabs(run.t["w2"]),
+                             k, cfg.score_fn, tokens=few)
+    y_few = O.bf16_to_f64(H.bf16_host(run.y[torch.from_numpy(few).cuda()]))
+    H.assert_close_out(y_few, y_def, f"{name} layer y")
