@@ -148,6 +148,75 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def stage_breakdown(cfg, t, reps=5):
+    """Per-stage device times of the unfused entry points and of the fused layer, cold L2
+    (a 512 MB buffer is overwritten before every timed call), with algorithmic bytes / flops."""
+    from paper_2605_05607_b200 import binding as B
+    shape = B.make_shape(cfg)
+    ws = B.alloc_workspace(shape)
+    T, E, k, d, f, P = cfg.T, cfg.E, cfg.k, cfg.d, cfg.f, cfg.P
+    dev = "cuda"
+    logits = torch.zeros(T * E, dtype=torch.float32, device=dev)
+    idx = torch.zeros(P, dtype=torch.int32, device=dev)
+    w = torch.zeros(P, dtype=torch.float32, device=dev)
+    lay = B.alloc_layout(shape)
+    xg = torch.zeros(T * min(k, cfg.G), d, dtype=torch.bfloat16, device=dev)
+    o = torch.zeros(P, d, dtype=torch.bfloat16, device=dev)
+    y = torch.zeros(T, d, dtype=torch.bfloat16, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+
+    calls = {
+        "route": lambda: B.moe_route(shape, t["x"], t["w_gate"], t["bias"], logits, idx, w, ws),
+        "layout": lambda: B.moe_dispatch(shape, t["x"], idx, lay, None, ws),
+        "dispatch": lambda: B.moe_dispatch(shape, t["x"], idx, lay, xg, ws),
+        "expert_ffn": lambda: B.moe_expert_ffn(shape, xg, lay, w, t["w1"], t["w3"], t["w2"], o, ws),
+        "combine": lambda: B.moe_combine(shape, o, lay, idx, w, None, y, ws),
+        "layer_fused": lambda: B.moe_layer(shape, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws),
+    }
+    kernels = {"route": ["gate", "topk"], "dispatch": ["dispatch"], "expert_ffn": ["gemm1", "gemm2"],
+               "combine": ["combine"]}
+    out = {}
+    for name, fn in calls.items():
+        fn()                                           # warm (and produces the next stage's input)
+        times = []
+        for _ in range(reps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        out[name] = {"ms": float(np.median(times))}
+        for kn in kernels.get(name, []):
+            B.moe_profile_enable(B.KERNEL_IDS[kn])
+            for _ in range(reps):
+                flush.fill_(1)
+                fn()
+            ms, n = B.moe_profile_read()
+            B.moe_profile_enable(0)
+            out[name][kn + "_kernel_ms"] = ms / max(n, 1)
+    n_disp = int(lay.group_offsets[cfg.G].item())
+    counts = lay.expert_counts[:E].cpu().numpy()
+    pk = peaks()
+    disp_bytes = (T + n_disp) * 2.0 * d
+    comb_bytes = (P + T) * 2.0 * d + 12.0 * P
+    flops = 6.0 * P * d * f
+    dk, ck = out["dispatch"]["dispatch_kernel_ms"], out["combine"]["combine_kernel_ms"]
+    g1, g2 = out["expert_ffn"]["gemm1_kernel_ms"], out["expert_ffn"]["gemm2_kernel_ms"]
+    out["dispatch"].update(bytes=disp_bytes, gbs=disp_bytes / dk / 1e6, frac_hbm_measured=disp_bytes / dk / 1e6 / pk["hbm_gbs"])
+    out["combine"].update(bytes=comb_bytes, gbs=comb_bytes / ck / 1e6, frac_hbm_measured=comb_bytes / ck / 1e6 / pk["hbm_gbs"])
+    out["expert_ffn"].update(flops=flops, tflops=flops / (g1 + g2) / 1e9,
+                             gemm1_tflops=4.0 * P * d * f / g1 / 1e9, gemm2_tflops=2.0 * P * d * f / g2 / 1e9,
+                             frac_bf16_sustained=flops / (g1 + g2) / 1e9 / pk["bf16_tflops_sustained"],
+                             frac_bf16_burst=flops / (g1 + g2) / 1e9 / pk["bf16_tflops"])
+    unfused = sum(out[n]["ms"] for n in ("route", "dispatch", "expert_ffn", "combine"))
+    out["summary"] = {"unfused_sum_ms": unfused, "fused_ms": out["layer_fused"]["ms"],
+                      "fused_tokens_per_s": T / out["layer_fused"]["ms"] * 1e3,
+                      "n_disp": n_disp, "pairs": P, "dedup": 1.0 - n_disp / P,
+                      "rows_per_expert_min": int(counts.min()), "rows_per_expert_max": int(counts.max()),
+                      "empty_experts": int((counts == 0).sum()), "timing": "cold L2 (512 MB overwrite before each call)"}
+    return out
+
+
 def workload_config(cfg, n_gpus):
     return {"workload": f"{cfg.name}: T={cfg.T} d={cfg.d} f={cfg.f} E={cfg.E} top-{cfg.k} G={cfg.G} per GPU",
             "T": cfg.T, "d": cfg.d, "f": cfg.f, "E": cfg.E, "k": cfg.k, "G": cfg.G,
@@ -167,6 +236,10 @@ def main():
     ap.add_argument("--ref-sample", type=int, default=0,
                     help="tokens per step of the reference arm (0: sized from a one-token calibration)")
     ap.add_argument("--cpu-sample", type=int, default=64, help="tokens of the cpu_baseline leg (0: skip)")
+    ap.add_argument("--lean", action="store_true",
+                    help="timed region only: no e2e / stage / cpu_baseline legs (for profiler captures)")
+    ap.add_argument("--report", default=None,
+                    help="also write per-stage numbers of every configuration to this JSON file (1 GPU)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "tcmoe" else args.warmup
     cfg = synth.CONFIGS[args.config]
@@ -231,29 +304,35 @@ def main():
     status = B.moe_status(ws)
     assert status[0] == 0, f"device status {status}"
 
-    # ---- end to end through the host-buffer entry point: pinned x in, y out, every step
-    x_host = t["x"].cpu().pin_memory()
-    y_host = torch.empty_like(x_host).pin_memory()
-    x_dev = torch.empty_like(t["x"])
-    for _ in range(3):
-        B.moe_layer_host(shape, x_host, x_dev, t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, y_host, ws)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
-        B.moe_layer_host(shape, x_host, x_dev, t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, y_host, ws)
-    e1.record()
-    barrier()
-    e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        tmax = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tmax.item())
+    e2e_ms = None
+    if not args.lean:
+        # ---- end to end through the host-buffer entry point: pinned x in, y out, every step
+        x_host = t["x"].cpu().pin_memory()
+        y_host = torch.empty_like(x_host).pin_memory()
+        x_dev = torch.empty_like(t["x"])
+
+        def step_host():
+            B.moe_layer_host(shape, x_host, x_dev, t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, y_host, ws)
+
+        for _ in range(3):
+            step_host()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.steps):
+            step_host()
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        if dist is not None:
+            tmax = torch.tensor([e2e_ms], device="cuda")
+            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+            e2e_ms = float(tmax.item())
 
     clocks = None
     if sampler is not None:
         clocks = sampler.summary(wall0, wall1)
-        if clocks["samples"] < 3:  # timed region too short for the 100 ms sampler: keep the same load running
+        if clocks["samples"] < 3 and not args.lean:  # timed region too short for the 100 ms sampler: keep the same load running
             p0 = time.time()
             while time.time() - p0 < 1.5:
                 for _ in range(10):
@@ -280,7 +359,8 @@ def main():
         "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic", "config": workload_config(cfg, world),
         "clocks": clocks,
-        "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.T * cfg.d * 2,
+        "e2e": None if e2e_ms is None else
+               {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.T * cfg.d * 2,
                 "d2h_bytes_per_step": cfg.T * cfg.d * 2},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": {"kernel": "ffn_gemm_kernel<0> (GEMM-1 + SwiGLU, tcgen05)", "bound": "tensor",
@@ -291,7 +371,22 @@ def main():
                      "traffic": GEMM1_DRAM_TRAFFIC.get(cfg.name)},
         "ffn_tflops_layer": 6.0 * cfg.P * cfg.d * cfg.f * args.steps / (elapsed_ms * 1e-3) / 1e12,
     }
-    if world == 1 and args.cpu_sample > 0:
+    if world == 1 and not args.lean:
+        line["stages"] = stage_breakdown(cfg, t)
+    if world == 1 and args.report and not args.lean:
+        report = {cfg.name: line["stages"]}
+        del t
+        torch.cuda.empty_cache()
+        for name, c in synth.CONFIGS.items():
+            if name != cfg.name:
+                tt = synth.make_inputs(c, "cuda")
+                report[name] = stage_breakdown(c, tt)
+                del tt
+                torch.cuda.empty_cache()
+        os.makedirs(os.path.dirname(os.path.abspath(args.report)), exist_ok=True)
+        json.dump({"peaks": pk, "configs": report}, open(args.report, "w"), indent=1)
+        t = synth.make_inputs(cfg, "cuda") if args.cpu_sample > 0 else None
+    if world == 1 and args.cpu_sample > 0 and not args.lean:
         dt, n = oracle_sample_run(cfg, t, args.cpu_sample)
         line["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                 "sample": f"{n} of {cfg.T} tokens, {dt:.1f} s (gate + top-k + expert FFN + combine)"}
