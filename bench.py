@@ -209,7 +209,26 @@ def stage_breakdown(cfg, t, reps=5):
                              frac_bf16_sustained=flops / (g1 + g2) / 1e9 / pk["bf16_tflops_sustained"],
                              frac_bf16_burst=flops / (g1 + g2) / 1e9 / pk["bf16_tflops"])
     unfused = sum(out[n]["ms"] for n in ("route", "dispatch", "expert_ffn", "combine"))
-    out["summary"] = {"unfused_sum_ms": unfused, "fused_ms": out["layer_fused"]["ms"],
+
+    # fused layer against the four unfused entry points issued back to back (same clocks, same
+    # power state: the two variants alternate)
+    def timed(fn):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); fn(); e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    def unfused_seq():
+        for n in ("route", "dispatch", "expert_ffn", "combine"):
+            calls[n]()
+
+    seq_ms, fus_ms = [], []
+    for _ in range(reps):
+        seq_ms.append(timed(unfused_seq))
+        fus_ms.append(timed(calls["layer_fused"]))
+    out["summary"] = {"unfused_sum_ms": unfused, "unfused_back_to_back_ms": float(np.median(seq_ms)),
+                      "fused_back_to_back_ms": float(np.median(fus_ms)), "fused_ms": out["layer_fused"]["ms"],
                       "fused_tokens_per_s": T / out["layer_fused"]["ms"] * 1e3,
                       "n_disp": n_disp, "pairs": P, "dedup": 1.0 - n_disp / P,
                       "rows_per_expert_min": int(counts.min()), "rows_per_expert_max": int(counts.max()),

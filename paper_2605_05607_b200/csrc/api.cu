@@ -14,7 +14,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Regions of the workspace, in order.  Every region starts on a 1 KiB boundary.
 struct WsPlan {
-  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, h, o, logits, topk_idx, topk_w;
+  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, h, o, logits, topk_idx, topk_w;
   size_t expert_counts, expert_offsets, group_counts, group_offsets, pair_row, row_pair, al, disp_token, row_src;
   size_t total;
   int W;
@@ -41,6 +41,7 @@ WsPlan plan(const moe_shape_t& s) {
   p.eprefix = take(E * W * 4);
   p.gprefix = take(G * W * 4);
   p.mt_prefix = take((E + 1) * 4);
+  p.mp_prefix = take((E + 1) * 4);
   p.h = take(P * (size_t)s.f * 2);
   p.o = take(P * (size_t)s.d * 2);
   p.logits = take(T * E * 4);
@@ -107,6 +108,7 @@ LayoutScratch scratch(void* ws, const WsPlan& p) {
   sc.eprefix = at<int32_t>(ws, p.eprefix);
   sc.gprefix = at<int32_t>(ws, p.gprefix);
   sc.mt_prefix = at<int32_t>(ws, p.mt_prefix);
+  sc.mp_prefix = at<int32_t>(ws, p.mp_prefix);
   sc.W = p.W;
   return sc;
 }
@@ -295,10 +297,11 @@ int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t*
   a.row_pair = layout->row_pair;
   a.expert_offsets = layout->expert_offsets;
   a.mt_prefix = at<int32_t>(ws, p.mt_prefix);
+  a.mp_prefix = at<int32_t>(ws, p.mp_prefix);
   a.status = at<int32_t>(ws, p.status);
   // rebuilt from the counts so that this call does not depend on what moe_dispatch left in ws
-  TCMOE_CUDA(launch_mt_prefix(to_shape(*shape), layout->expert_counts, at<int32_t>(ws, p.mt_prefix),
-                              static_cast<cudaStream_t>(stream)));
+  TCMOE_CUDA(launch_tile_prefix(to_shape(*shape), layout->expert_counts, at<int32_t>(ws, p.mt_prefix),
+                                at<int32_t>(ws, p.mp_prefix), static_cast<cudaStream_t>(stream)));
   TCMOE_CUDA(launch_expert_ffn(to_shape(*shape), a, static_cast<cudaStream_t>(stream)));
   return MOE_OK;
 }
@@ -368,6 +371,7 @@ int moe_layer(const moe_shape_t* shape, const void* x, const float* w_gate, cons
   a.row_pair = L.row_pair;
   a.expert_offsets = L.expert_offsets;
   a.mt_prefix = at<int32_t>(ws, p.mt_prefix);
+  a.mp_prefix = at<int32_t>(ws, p.mp_prefix);
   a.status = status;
   TCMOE_CUDA(launch_expert_ffn(s, a, st));
   TCMOE_CUDA(launch_combine(s, a.o, L, idx, tw, nullptr, y, st));

@@ -37,7 +37,8 @@ struct LayoutScratch {
   uint32_t* gmask;    // [G, W] token t touches group g
   int32_t* eprefix;   // [E, W] exclusive popcount prefix along the row
   int32_t* gprefix;   // [G, W]
-  int32_t* mt_prefix; // [E+1]  exclusive prefix of 128-row tiles per expert
+  int32_t* mt_prefix; // [E+1]  exclusive prefix of 128-row tiles per expert (GEMM-1 tasks)
+  int32_t* mp_prefix; // [E+1]  exclusive prefix of 256-row CTA-pair tiles per expert (GEMM-2 tasks)
   int W;
 };
 
@@ -48,7 +49,8 @@ cudaError_t launch_topk(const Shape& s, const float* logits, const float* bias, 
 // layout.cu
 cudaError_t launch_layout(const Shape& s, const int32_t* topk_idx, const Layout& L, const LayoutScratch& sc,
                           int32_t* status, cudaStream_t st);
-cudaError_t launch_mt_prefix(const Shape& s, const int32_t* expert_counts, int32_t* mt_prefix, cudaStream_t st);
+cudaError_t launch_tile_prefix(const Shape& s, const int32_t* expert_counts, int32_t* mt_prefix, int32_t* mp_prefix,
+                               cudaStream_t st);
 cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void* xg, cudaStream_t st);
 cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
                            const float* topk_w, void* pg, void* y, cudaStream_t st);
@@ -63,7 +65,8 @@ struct FfnArgs {
   const float* topk_w;        // NULL: un-weighted epilogue
   const int32_t* row_pair;
   const int32_t* expert_offsets;
-  const int32_t* mt_prefix;
+  const int32_t* mt_prefix;   // 128-row tiles per expert, exclusive prefix
+  const int32_t* mp_prefix;   // 256-row pair tiles per expert, exclusive prefix
   int32_t* status;
 };
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st);

@@ -1,0 +1,91 @@
+// Pieces shared by the two expert-FFN GEMM kernels (paper Sec. II-A GEMM-1 / GEMM-2): tile
+// geometry, the device-side task decode, UMMA descriptors and small epilogue helpers.
+#pragma once
+#include "common.cuh"
+#include "ptx.cuh"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+namespace tcmoe {
+namespace ffn {
+
+constexpr int BM = 128;       // rows per CTA tile (the paper's tsize: 128-token tiles, Sec. VI-H)
+constexpr int BK = 64;        // K per pipeline stage = one 128-byte swizzle row of bf16
+constexpr int UMMA_N = 256;   // accumulator columns per tile
+constexpr int MAX_E = 1024;
+
+struct GemmParams {
+  const __nv_bfloat16* a_src;   // GEMM-1 gather source (xg or x)
+  int a_ld;
+  const int32_t* gather_idx;    // row_src, or row_pair with gather_div = k (token = row_pair / k)
+  int gather_div;
+  __nv_bfloat16* out;
+  int out_ld;
+  const float* topk_w;          // GEMM-2 epilogue weights (NULL: 1)
+  const int32_t* row_pair;
+  const int32_t* expert_offsets;
+  const int32_t* tile_prefix;   // exclusive prefix of tiles per expert (128-row tiles for GEMM-1,
+                                // 256-row CTA-pair tiles for GEMM-2)
+  int E, K, N, n_tiles;
+  int32_t* status;
+};
+
+struct Tile {
+  int e, n0, row0, rows;
+};
+
+// Task w -> (expert, n-tile, m-tile), ordered expert-major, then n-tile, m-tile fastest so that
+// CTAs running at the same time share the weight tile in L2.  `rows_per_tile` is 128 (one CTA) or
+// 256 (a CTA pair; CTA `rank` owns the rank-th half).  rows <= 0: nothing of this CTA is valid.
+__device__ __forceinline__ Tile decode_tile(int w, const int* tp, const int* eoff, int E, int n_tiles, int bn_out,
+                                            int rows_per_tile, int rank) {
+  int lo = 0, hi = E;  // tp[lo] * n_tiles <= w < tp[hi] * n_tiles
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (tp[mid] * n_tiles <= w) lo = mid; else hi = mid;
+  }
+  const int local = w - tp[lo] * n_tiles;
+  const int mt = tp[lo + 1] - tp[lo];
+  Tile t;
+  t.e = lo;
+  t.n0 = (local / mt) * bn_out;
+  t.row0 = eoff[lo] + (local % mt) * rows_per_tile + rank * BM;
+  t.rows = min(BM, eoff[lo + 1] - t.row0);
+  return t;
+}
+
+// 64-bit shared-memory matrix descriptors (sm_100 format: version 1, 128-byte swizzle).
+//  A, K-major : rows of 128 B; 8-row groups 1024 B apart (SBO); LBO unused.
+//  B, MN-major: 64-column slabs; inside a slab 8 K-rows of 128 B form a 1024-B atom, atoms of
+//               successive K 1024 B apart (SBO); slabs BK*128 B apart (LBO).
+__device__ __forceinline__ uint64_t desc_base(uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return ((uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16) | ((uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+__device__ __forceinline__ uint64_t desc_at(uint64_t base, uint32_t smem_addr) {
+  return base | (uint64_t)((smem_addr & 0x3FFFF) >> 4);
+}
+
+// instruction descriptor: D fp32, A/B bf16, A K-major, B MN-major, N = 256, M = m
+__host__ __device__ constexpr uint32_t idesc_bf16(int m) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((uint32_t)(UMMA_N >> 3) << 17) |
+         ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ float silu_mul(float a, float b) { return __fdividef(a, 1.f + __expf(-a)) * b; }
+
+__device__ __forceinline__ uint32_t pack2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, cudaStream_t st);
+cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, cudaStream_t st);
+
+}  // namespace ffn
+}  // namespace tcmoe

@@ -1,0 +1,272 @@
+// GEMM-1 of the expert FFN with the SwiGLU epilogue (paper Sec. II-A "GEMM-1"; Sec. IV: the
+// dispatch gather is the GEMM's prologue, tiles of 128 tokens):
+//     h[r, n] = silu(a_r . W1[e][:, n]) * (a_r . W3[e][:, n]),   a_r = src[gather_idx[r] / gather_div]
+//
+// A rows are GATHERED (they are arbitrary rows of the dispatched buffer, or of x itself in the
+// fused layer) by cp.async into the 128-byte swizzled K-major layout the UMMA descriptor expects;
+// B = two 64-column slabs of W1 and the same two of W3 loaded by TMA side by side, so that ONE
+// 128 x 256 x 16 UMMA yields both products (accumulator columns [0,128) = a.W1, [128,256) = a.W3).
+//
+// One persistent CTA per SM (tcgen05 cta_group::1) walks tile tasks decoded from the device-side
+// tile prefix, so no routing-dependent quantity visits the host.  Warp roles: 0-3 epilogue
+// (TMEM -> registers -> SwiGLU -> global), 4 TMA producer, 5 UMMA issuer and TMEM owner, 6-9 gather
+// producers.  Accumulators are double-buffered in TMEM (2 x 256 columns): the epilogue of tile i
+// overlaps the main loop of tile i+1.  Every wait is bounded.
+//
+// A CTA-pair (cta_group::2) variant of this kernel was measured slower: with the UMMA twice as
+// fast per CTA the gather -> fence -> arrive -> UMMA chain of the peer CTA no longer fits the
+// pipeline depth, and TMA tile::gather4 sustains only one 4-row instruction per ~40 ns.
+#include "ffn_common.cuh"
+
+namespace tcmoe {
+namespace ffn {
+namespace {
+
+constexpr int NSTAGE = 4;
+constexpr int A_BYTES = BM * BK * 2;         // 16 KiB
+constexpr int B_BYTES = UMMA_N * BK * 2;     // 32 KiB = four 64-column slabs of 8 KiB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int GATHER_LAG = 2;                // cp.async groups kept in flight per gather thread
+constexpr int NUM_BARS = 2 * NSTAGE + 4;
+constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + 2 * (MAX_E + 1) * 4;
+constexpr int THREADS = 320;
+constexpr int BN_OUT = 128;
+constexpr uint32_t IDESC = idesc_bf16(BM);
+
+__global__ void __launch_bounds__(THREADS, 1)
+ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w3,
+                 const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + NSTAGE * STAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
+  int* abort_s = reinterpret_cast<int*>(tmem_slot + 1);
+  int* tp_s = reinterpret_cast<int*>(tmem_slot + 16);
+  int* eoff_s = tp_s + (MAX_E + 1);
+
+  const uint32_t smem_base = ptx::smem_u32(smem);
+  const uint32_t bar_base = ptx::smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (NSTAGE + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * NSTAGE + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * NSTAGE + 2 + b); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  for (int i = threadIdx.x; i <= p.E; i += blockDim.x) {
+    tp_s[i] = p.tile_prefix[i];
+    eoff_s[i] = p.expert_offsets[i];
+  }
+  if (threadIdx.x == 0) {
+    *abort_s = p.status[ST_ABORT];
+    for (int s = 0; s < NSTAGE; ++s) {
+      ptx::mbar_init(full_bar(s), 1 + 4);   // TMA thread + one lane per gather warp
+      ptx::mbar_init(empty_bar(s), 1);      // tcgen05.commit
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(tfull_bar(b), 1);      // tcgen05.commit
+      ptx::mbar_init(tempty_bar(b), 4);     // one lane per epilogue warp
+    }
+    ptx::fence_mbar_init();
+  }
+  if (warp == 4 && lane == 0) {
+    ptx::prefetch_tensormap(&map_w1);
+    ptx::prefetch_tensormap(&map_w3);
+  }
+  if (warp == 5) {
+    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int total = tp_s[p.E] * p.n_tiles;
+  const int KB = (p.K + BK - 1) / BK;
+  volatile int* abort_flag = abort_s;
+  const volatile int* global_abort = p.status + ST_ABORT;
+
+  auto timeout = [&](int detail) {
+    report_error(p.status, DEV_TIMEOUT, KID_GEMM1, detail, blockIdx.x);
+    p.status[ST_ABORT] = 1;
+    *abort_flag = 1;
+  };
+  auto tile_of = [&](int w) { return decode_tile(w, tp_s, eoff_s, p.E, p.n_tiles, BN_OUT, BM, 0); };
+
+  if (warp < 4) {
+    // ================================ epilogue ================================
+    int tl = 0;
+    for (int w = blockIdx.x; w < total && !*abort_flag; w += gridDim.x, ++tl) {
+      const Tile t = tile_of(w);
+      const int buf = tl & 1;
+      if (!ptx::mbar_wait_warp<true>(tfull_bar(buf), (tl >> 1) & 1, abort_flag, global_abort)) { timeout(1); break; }
+      ptx::tc_fence_after();
+      const int lrow = warp * 32 + lane;
+      const bool valid = lrow < t.rows;
+      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UMMA_N);
+      __nv_bfloat16* orow = p.out + (size_t)(valid ? t.row0 + lrow : 0) * (size_t)p.out_ld + t.n0;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        uint32_t a1[32], a3[32];
+        ptx::tmem_ld32(taddr + c * 32, a1);
+        ptx::tmem_ld32(taddr + 128 + c * 32, a3);
+        ptx::tmem_ld_wait();
+        if (valid) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            if (t.n0 + c * 32 + v * 8 < p.N) {
+              uint4 q;
+              uint32_t* qq = reinterpret_cast<uint32_t*>(&q);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int j = v * 8 + 2 * i;
+                qq[i] = pack2(silu_mul(__uint_as_float(a1[j]), __uint_as_float(a3[j])),
+                              silu_mul(__uint_as_float(a1[j + 1]), __uint_as_float(a3[j + 1])));
+              }
+              *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = q;
+            }
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
+    }
+  } else if (warp == 4) {
+    // ================================ TMA producer (weights) ================================
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int w = blockIdx.x; w < total && !*abort_flag; w += gridDim.x) {
+        const Tile t = tile_of(w);
+        bool ok = true;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % NSTAGE;
+          if (!ptx::mbar_wait(empty_bar(s), ((it / NSTAGE) & 1) ^ 1, abort_flag, global_abort)) {
+            timeout(2); ok = false; break;
+          }
+          const uint32_t sb = smem_base + s * STAGE_BYTES + A_BYTES;
+          ptx::mbar_arrive_expect_tx(full_bar(s), B_BYTES);
+          const int k0 = kb * BK;
+          ptx::tma_load_3d(sb, &map_w1, full_bar(s), t.n0, k0, t.e);
+          ptx::tma_load_3d(sb + 8192, &map_w1, full_bar(s), t.n0 + 64, k0, t.e);
+          ptx::tma_load_3d(sb + 16384, &map_w3, full_bar(s), t.n0, k0, t.e);
+          ptx::tma_load_3d(sb + 24576, &map_w3, full_bar(s), t.n0 + 64, k0, t.e);
+        }
+        if (!ok) break;
+      }
+    }
+  } else if (warp == 5) {
+    // ================================ UMMA issuer ================================
+    if (lane == 0) {
+      const uint64_t a_base = desc_base(16, 1024);
+      const uint64_t b_base = desc_base(BK * 128, 1024);
+      uint32_t it = 0;
+      int tl = 0;
+      for (int w = blockIdx.x; w < total && !*abort_flag; w += gridDim.x, ++tl) {
+        const int buf = tl & 1;
+        if (!ptx::mbar_wait(tempty_bar(buf), ((tl >> 1) & 1) ^ 1, abort_flag, global_abort)) { timeout(3); break; }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * UMMA_N);
+        bool ok = true;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % NSTAGE;
+          if (!ptx::mbar_wait(full_bar(s), (it / NSTAGE) & 1, abort_flag, global_abort)) {
+            timeout(4); ok = false; break;
+          }
+          ptx::tc_fence_after();
+          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+          const uint64_t ad = desc_at(a_base, sa), bd = desc_at(b_base, sb);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)  // K = 16 per UMMA: A +32 B inside the swizzle row, B +2 atoms
+            ptx::umma_bf16(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), IDESC, (kb | k) != 0);
+          ptx::umma_commit(empty_bar(s));   // frees the stage when these UMMAs have read it
+        }
+        if (!ok) break;
+        ptx::umma_commit(tfull_bar(buf));   // accumulator complete
+      }
+    }
+  } else {
+    // ================================ A gather producers ================================
+    const int gt = threadIdx.x - 192;     // 0..127
+    const int chunk = gt & 7;             // 16-byte chunk of the 128-byte K row
+    const int rbase = gt >> 3;            // rows rbase + 16 j
+    uint32_t it = 0;
+    for (int w = blockIdx.x; w < total && !*abort_flag; w += gridDim.x) {
+      const Tile t = tile_of(w);
+      const __nv_bfloat16* src[8];
+      uint32_t live = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int lr = rbase + 16 * j;
+        src[j] = p.a_src;
+        if (lr < t.rows) {
+          int idx = __ldg(p.gather_idx + t.row0 + lr);
+          if (p.gather_div > 1) idx /= p.gather_div;
+          src[j] = p.a_src + (size_t)idx * p.a_ld;
+          live |= 1u << j;
+        }
+      }
+      bool ok = true;
+      for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int s = it % NSTAGE;
+        if (!ptx::mbar_wait(empty_bar(s), ((it / NSTAGE) & 1) ^ 1, abort_flag, global_abort)) {
+          timeout(5); ok = false; break;
+        }
+        const uint32_t sa = smem_base + s * STAGE_BYTES;
+        const int col = kb * BK + chunk * 8;
+        const bool kin = col < p.K;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int lr = rbase + 16 * j;
+          const uint32_t dst = sa + lr * 128 + ((chunk ^ (lr & 7)) << 4);
+          const bool on = kin && ((live >> j) & 1u);
+          ptx::cp_async_16(dst, on ? (const void*)(src[j] + col) : (const void*)p.a_src, on ? 16u : 0u);
+        }
+        ptx::cp_async_commit();
+        if (it >= GATHER_LAG) {
+          ptx::cp_async_wait<GATHER_LAG>();
+          ptx::fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(full_bar((it - GATHER_LAG) % NSTAGE));
+        }
+      }
+      if (!ok) break;
+    }
+    ptx::cp_async_wait<0>();
+    ptx::fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+      const uint32_t first = it >= GATHER_LAG ? it - GATHER_LAG : 0;
+      for (uint32_t i = first; i < it; ++i) ptx::mbar_arrive(full_bar(i % NSTAGE));
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // abort path only: give bulk copies still in flight time to land before the CTA retires
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+  }
+  __syncthreads();
+  if (warp == 5) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  ProfileScope prof(KID_GEMM1, st);
+  ffn_gemm1_kernel<<<sm_count(), THREADS, SMEM_BYTES, st>>>(m_w1, m_w3, p);
+  return cudaGetLastError();
+}
+
+}  // namespace ffn
+}  // namespace tcmoe

@@ -1,0 +1,254 @@
+// GEMM-2 of the expert FFN with the gate weight in the epilogue (paper Sec. II-A "GEMM-2";
+// Sec. III-C: expert i scales its output by w_i in GEMM-2's epilogue so that Combine can be an
+// un-weighted reduction):
+//     o[r, n] = w_r * (h_r . W2[e][:, n])
+//
+// Both operands come by TMA (h rows are contiguous in expert-sorted order).  CTAs work in pairs
+// (cluster of 2, tcgen05 cta_group::2): each CTA holds 128 rows of h and one half of the
+// 256-column W2 tile; one UMMA of M = 256 spans the pair, so every weight byte is fetched and read
+// from shared memory once per 256 rows.  Rank 0 of the pair (the leader) issues every UMMA.
+//
+// Barrier ownership in a pair:
+//   full[s]    leader's copy: the leader announces the bytes of both CTAs, both CTAs' TMA loads
+//              credit it
+//   empty[s]   each CTA's own copy, signalled by the leader's tcgen05.commit (one commit per CTA)
+//   tfull[b]   each CTA's own copy (accumulator buffer b complete), same
+//   tempty[b]  leader's copy: the 4 epilogue warps of each CTA arrive when buffer b is drained
+//
+// Warp roles: 0-3 epilogue, 4 TMA producer, 5 UMMA issuer (leader only) and TMEM owner.
+// Accumulators are double-buffered in TMEM; every wait is bounded; neither CTA retires before its
+// peer has stopped touching its shared memory and TMEM (cluster barrier at the end).
+#include "ffn_common.cuh"
+
+namespace tcmoe {
+namespace ffn {
+namespace {
+
+constexpr int NSTAGE = 6;
+constexpr int A_BYTES = BM * BK * 2;            // 16 KiB: this CTA's 128 rows
+constexpr int B_BYTES = (UMMA_N / 2) * BK * 2;  // 16 KiB: this CTA's half of the B tile (two 64-column slabs)
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int NUM_BARS = 2 * NSTAGE + 4;
+constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + 2 * (MAX_E + 1) * 4;
+constexpr int THREADS = 192;
+constexpr int BN_OUT = 256;
+constexpr uint32_t IDESC = idesc_bf16(2 * BM);
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_h,
+                 const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + NSTAGE * STAGE_BYTES);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
+  int* abort_s = reinterpret_cast<int*>(tmem_slot + 1);
+  int* tp_s = reinterpret_cast<int*>(tmem_slot + 16);
+  int* eoff_s = tp_s + (MAX_E + 1);
+
+  const uint32_t smem_base = ptx::smem_u32(smem);
+  const uint32_t bar_base = ptx::smem_u32(bars);
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (NSTAGE + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * NSTAGE + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * NSTAGE + 2 + b); };
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rank = (int)ptx::cluster_ctarank();
+  const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
+
+  for (int i = threadIdx.x; i <= p.E; i += blockDim.x) {
+    tp_s[i] = p.tile_prefix[i];
+    eoff_s[i] = p.expert_offsets[i];
+  }
+  if (threadIdx.x == 0) {
+    *abort_s = p.status[ST_ABORT];
+    for (int s = 0; s < NSTAGE; ++s) {
+      ptx::mbar_init(full_bar(s), 1);       // leader TMA thread (expect_tx for both CTAs)
+      ptx::mbar_init(empty_bar(s), 1);      // tcgen05.commit
+    }
+    for (int b = 0; b < 2; ++b) {
+      ptx::mbar_init(tfull_bar(b), 1);      // tcgen05.commit
+      ptx::mbar_init(tempty_bar(b), 8);     // one lane per epilogue warp, both CTAs
+    }
+    ptx::fence_mbar_init();
+  }
+  if (warp == 4 && lane == 0) {
+    ptx::prefetch_tensormap(&map_w2);
+    ptx::prefetch_tensormap(&map_h);
+  }
+  if (warp == 5) {
+    ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), 512);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync();   // the peer's barriers are initialised before anything signals them
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int total = tp_s[p.E] * p.n_tiles;
+  const int KB = (p.K + BK - 1) / BK;
+  volatile int* abort_flag = abort_s;
+  const volatile int* global_abort = p.status + ST_ABORT;
+
+  auto timeout = [&](int detail) {
+    report_error(p.status, DEV_TIMEOUT, KID_GEMM2, detail, blockIdx.x);
+    p.status[ST_ABORT] = 1;
+    *abort_flag = 1;
+  };
+  auto tile_of = [&](int w) { return decode_tile(w, tp_s, eoff_s, p.E, p.n_tiles, BN_OUT, 2 * BM, rank); };
+
+  if (warp < 4) {
+    // ================================ epilogue (both CTAs) ================================
+    int tl = 0;
+    for (int w = cluster_id; w < total && !*abort_flag; w += num_clusters, ++tl) {
+      const Tile t = tile_of(w);
+      const int buf = tl & 1;
+      if (!ptx::mbar_wait_warp<true>(tfull_bar(buf), (tl >> 1) & 1, abort_flag, global_abort)) { timeout(1); break; }
+      ptx::tc_fence_after();
+      const int lrow = warp * 32 + lane;
+      const bool valid = lrow < t.rows;
+      const size_t grow = (size_t)(valid ? t.row0 + lrow : 0);
+      const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UMMA_N);
+      __nv_bfloat16* orow = p.out + grow * (size_t)p.out_ld + t.n0;
+      float wr = 1.f;
+      if (valid && p.topk_w != nullptr) wr = __ldg(p.topk_w + __ldg(p.row_pair + grow));
+#pragma unroll 1
+      for (int c = 0; c < 8; ++c) {
+        uint32_t acc[32];
+        ptx::tmem_ld32(taddr + c * 32, acc);
+        ptx::tmem_ld_wait();
+        if (valid) {
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            if (t.n0 + c * 32 + v * 8 < p.N) {
+              uint4 q;
+              uint32_t* qq = reinterpret_cast<uint32_t*>(&q);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int j = v * 8 + 2 * i;
+                qq[i] = pack2(wr * __uint_as_float(acc[j]), wr * __uint_as_float(acc[j + 1]));
+              }
+              *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = q;
+            }
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(buf), 0));
+    }
+  } else if (warp == 4) {
+    // ================================ TMA producer (both CTAs) ================================
+    if (lane == 0) {
+      uint32_t it = 0;
+      for (int w = cluster_id; w < total && !*abort_flag; w += num_clusters) {
+        const Tile t = tile_of(w);
+        bool ok = true;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % NSTAGE;
+          if (!ptx::mbar_wait(empty_bar(s), ((it / NSTAGE) & 1) ^ 1, abort_flag, global_abort)) {
+            timeout(2); ok = false; break;
+          }
+          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+          const uint32_t lead_full = ptx::mapa(full_bar(s), 0);
+          // the leader announces the bytes of both CTAs; the peer's copies only complete them
+          if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+          const int k0 = kb * BK;
+          ptx::tma_load_2d_pair(sa, &map_h, lead_full, k0, t.row0);
+          ptx::tma_load_3d_pair(sb, &map_w2, lead_full, t.n0 + rank * 128, k0, t.e);
+          ptx::tma_load_3d_pair(sb + 8192, &map_w2, lead_full, t.n0 + rank * 128 + 64, k0, t.e);
+        }
+        if (!ok) break;
+      }
+    }
+  } else if (warp == 5) {
+    // ================================ UMMA issuer (leader CTA only) ================================
+    if (rank == 0 && lane == 0) {
+      const uint64_t a_base = desc_base(16, 1024);
+      const uint64_t b_base = desc_base(BK * 128, 1024);
+      uint32_t it = 0;
+      int tl = 0;
+      for (int w = cluster_id; w < total && !*abort_flag; w += num_clusters, ++tl) {
+        const int buf = tl & 1;
+        if (!ptx::mbar_wait_cluster(tempty_bar(buf), ((tl >> 1) & 1) ^ 1, abort_flag, global_abort)) {
+          timeout(3); break;
+        }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * UMMA_N);
+        bool ok = true;
+        for (int kb = 0; kb < KB; ++kb, ++it) {
+          const int s = it % NSTAGE;
+          if (!ptx::mbar_wait_cluster(full_bar(s), (it / NSTAGE) & 1, abort_flag, global_abort)) {
+            timeout(4); ok = false; break;
+          }
+          ptx::tc_fence_after();
+          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
+          const uint64_t ad = desc_at(a_base, sa), bd = desc_at(b_base, sb);
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k)  // K = 16 per UMMA: A +32 B inside the swizzle row, B +2 atoms
+            ptx::umma_bf16_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), IDESC, (kb | k) != 0);
+          // free the stage in both CTAs once these UMMAs have read it
+          ptx::umma_commit_pair(ptx::mapa(empty_bar(s), 0));
+          ptx::umma_commit_pair(ptx::mapa(empty_bar(s), 1));
+        }
+        if (!ok) break;
+        ptx::umma_commit_pair(ptx::mapa(tfull_bar(buf), 0));   // accumulator complete, both halves
+        ptx::umma_commit_pair(ptx::mapa(tfull_bar(buf), 1));
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag || *global_abort) {
+    // abort path only: give bulk copies still in flight time to land before the CTAs retire
+    for (int i = 0; i < 64; ++i) __nanosleep(1000);
+  }
+  ptx::cluster_sync();   // neither CTA leaves while its peer may still touch its shared memory / TMEM
+  if (warp == 5) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(tmem_base, 512);
+  }
+}
+
+// Persistent grid: two CTAs per resident cluster, at most one CTA per SM.
+int pair_grid() {
+  static int g = 0;
+  if (g == 0) {
+    int clusters = 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(sm_count() & ~1);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    if (cudaOccupancyMaxActiveClusters(&clusters, ffn_gemm2_kernel, &cfg) != cudaSuccess || clusters <= 0) {
+      (void)cudaGetLastError();
+      clusters = sm_count() / 2;
+    }
+    g = 2 * min(clusters, sm_count() / 2);
+  }
+  return g;
+}
+
+}  // namespace
+
+cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  ProfileScope prof(KID_GEMM2, st);
+  ffn_gemm2_kernel<<<pair_grid(), THREADS, SMEM_BYTES, st>>>(m_w2, m_h, p);
+  return cudaGetLastError();
+}
+
+}  // namespace ffn
+}  // namespace tcmoe

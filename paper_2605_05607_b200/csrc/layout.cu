@@ -74,29 +74,30 @@ __global__ void __launch_bounds__(256) scan_masks_kernel(const uint32_t* __restr
   }
 }
 
-// ---- K2c: offsets (exclusive scans over experts / groups) and the 128-row tile prefix -----------
+// ---- K2c: offsets (exclusive scans over experts / groups) and the GEMM tile prefixes --------------
 __global__ void __launch_bounds__(1024) offsets_kernel(const int32_t* __restrict__ expert_counts,
                                                        const int32_t* __restrict__ group_counts,
                                                        int32_t* expert_offsets, int32_t* group_offsets,
-                                                       int32_t* mt_prefix, int E, int G) {
-  __shared__ int buf[3][1024];
+                                                       int32_t* mt_prefix, int32_t* mp_prefix, int E, int G) {
+  __shared__ int buf[4][1024];
   const int i = threadIdx.x;
   const int ce = (i < E) ? expert_counts[i] : 0;
   const int cg = (i < G) ? group_counts[i] : 0;
   buf[0][i] = ce;
   buf[1][i] = cg;
-  buf[2][i] = (ce + 127) >> 7;
+  buf[2][i] = (ce + 127) >> 7;   // 128-row tiles (GEMM-1)
+  buf[3][i] = (ce + 255) >> 8;   // 256-row CTA-pair tiles (GEMM-2)
   __syncthreads();
   for (int off = 1; off < 1024; off <<= 1) {  // Hillis-Steele inclusive scan, three lanes at once
-    int a = 0, b = 0, c = 0;
-    if (i >= off) { a = buf[0][i - off]; b = buf[1][i - off]; c = buf[2][i - off]; }
+    int a = 0, b = 0, c = 0, d = 0;
+    if (i >= off) { a = buf[0][i - off]; b = buf[1][i - off]; c = buf[2][i - off]; d = buf[3][i - off]; }
     __syncthreads();
-    buf[0][i] += a; buf[1][i] += b; buf[2][i] += c;
+    buf[0][i] += a; buf[1][i] += b; buf[2][i] += c; buf[3][i] += d;
     __syncthreads();
   }
-  if (i < E) { expert_offsets[i + 1] = buf[0][i]; mt_prefix[i + 1] = buf[2][i]; }
+  if (i < E) { expert_offsets[i + 1] = buf[0][i]; mt_prefix[i + 1] = buf[2][i]; mp_prefix[i + 1] = buf[3][i]; }
   if (i < G) group_offsets[i + 1] = buf[1][i];
-  if (i == 0) { expert_offsets[0] = 0; group_offsets[0] = 0; mt_prefix[0] = 0; }
+  if (i == 0) { expert_offsets[0] = 0; group_offsets[0] = 0; mt_prefix[0] = 0; mp_prefix[0] = 0; }
 }
 
 // ---- K2d: ranks -> row tables ----------------------------------------------------------------
@@ -129,25 +130,29 @@ __global__ void __launch_bounds__(256) fill_layout_kernel(const int32_t* __restr
   }
 }
 
-// exclusive prefix of 128-row tiles per expert, from the counts alone
-__global__ void __launch_bounds__(1024) mt_prefix_kernel(const int32_t* __restrict__ expert_counts,
-                                                         int32_t* mt_prefix, int E) {
-  __shared__ int buf[1024];
+// exclusive prefixes of 128-row tiles and 256-row pair tiles per expert, from the counts alone
+__global__ void __launch_bounds__(1024) tile_prefix_kernel(const int32_t* __restrict__ expert_counts,
+                                                           int32_t* mt_prefix, int32_t* mp_prefix, int E) {
+  __shared__ int buf[2][1024];
   const int i = threadIdx.x;
-  buf[i] = (i < E) ? (expert_counts[i] + 127) >> 7 : 0;
+  const int c = (i < E) ? expert_counts[i] : 0;
+  buf[0][i] = (c + 127) >> 7;
+  buf[1][i] = (c + 255) >> 8;
   __syncthreads();
   for (int off = 1; off < 1024; off <<= 1) {
-    const int a = (i >= off) ? buf[i - off] : 0;
+    int a = 0, b = 0;
+    if (i >= off) { a = buf[0][i - off]; b = buf[1][i - off]; }
     __syncthreads();
-    buf[i] += a;
+    buf[0][i] += a; buf[1][i] += b;
     __syncthreads();
   }
-  if (i < E) mt_prefix[i + 1] = buf[i];
-  if (i == 0) mt_prefix[0] = 0;
+  if (i < E) { mt_prefix[i + 1] = buf[0][i]; mp_prefix[i + 1] = buf[1][i]; }
+  if (i == 0) { mt_prefix[0] = 0; mp_prefix[0] = 0; }
 }
 
-cudaError_t launch_mt_prefix(const Shape& s, const int32_t* expert_counts, int32_t* mt_prefix, cudaStream_t st) {
-  mt_prefix_kernel<<<1, 1024, 0, st>>>(expert_counts, mt_prefix, s.E);
+cudaError_t launch_tile_prefix(const Shape& s, const int32_t* expert_counts, int32_t* mt_prefix, int32_t* mp_prefix,
+                               cudaStream_t st) {
+  tile_prefix_kernel<<<1, 1024, 0, st>>>(expert_counts, mt_prefix, mp_prefix, s.E);
   return cudaGetLastError();
 }
 
@@ -162,7 +167,7 @@ cudaError_t launch_layout(const Shape& s, const int32_t* topk_idx, const Layout&
   scan_masks_kernel<<<s.E + s.G, 256, 0, st>>>(sc.emask, sc.gmask, sc.eprefix, sc.gprefix, L.expert_counts,
                                                 L.group_counts, s.E, sc.W);
   offsets_kernel<<<1, 1024, 0, st>>>(L.expert_counts, L.group_counts, L.expert_offsets, L.group_offsets,
-                                     sc.mt_prefix, s.E, s.G);
+                                     sc.mt_prefix, sc.mp_prefix, s.E, s.G);
   if (s.T > 0) fill_layout_kernel<<<tb, 256, 0, st>>>(topk_idx, L, sc, s.T, s.E, s.k, s.G, m);
   return cudaGetLastError();
 }
