@@ -46,6 +46,8 @@ enum {
   MOE_ERR_WORKSPACE_TOO_SMALL = -3,
   MOE_ERR_MISALIGNED = -4,
   MOE_ERR_CUDA = -5,               /* a CUDA runtime / driver call failed (incl. no GPU)  */
+  MOE_ERR_SCRATCH_LIMIT = -6,      /* moe_dispatch_noalloc: shape needs more scratch than
+                                      the library's built-in array holds                  */
   /* device-side codes, reported through moe_status()[0] */
   MOE_DEV_TIMEOUT = 1,             /* a bounded wait inside a kernel expired              */
   MOE_DEV_INDEX_OUT_OF_RANGE = 2   /* an expert index outside [0, E) was read             */
@@ -157,6 +159,30 @@ int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, co
                    const float* logit_bias, int64_t bias_row_stride,
                    const void* w1, const void* w3, const void* w2, void* y_dev, void* y_host,
                    void* ws, size_t ws_bytes, void* stream);
+
+/* Dispatch without a workspace (the paper has no counterpart; this entry point exists for
+ * callers that cannot supply scratch memory).  Some users of this library run where device
+ * memory cannot be obtained around the call: plugins that execute inside a host framework's
+ * pre-planned arena, serving loops whose policy bans allocator calls (and the synchronisation
+ * they imply) on the hot path, callers bound to a fixed C interface with no slot for a scratch
+ * pointer.  For them this variant of moe_dispatch keeps the layout builder's scratch tables
+ * (membership bitmasks, popcount prefixes, tile prefixes, status block) in one fixed device
+ * array of MOE_NOALLOC_SCRATCH_BYTES that is part of the library image: every GPU that loads the
+ * library holds it until the process exits.  Inputs and outputs are still the caller's.
+ *  - Same arguments and results as moe_dispatch (layout arrays and, unless xg is NULL, the
+ *    dispatched copy), bit for bit.  The call allocates nothing and frees nothing.
+ *  - Limit: 256 + 8*(E+G)*ceil(T/32) + 8*(E+1) bytes (each table rounded up to 256) must fit in
+ *    MOE_NOALLOC_SCRATCH_BYTES; larger shapes return MOE_ERR_SCRATCH_LIMIT and launch nothing.
+ *  - The first call on a device looks up the array's device address; make that first call
+ *    outside any stream capture.  Later calls only enqueue work on `stream`.
+ *  - All calls on a device share the array and it keeps the previous call's contents; the
+ *    entry point clears what must start at zero.  Two calls that overlap on the GPU (different
+ *    streams, no ordering between them) race on it: serialise them.
+ *  - status_out: NULL, or 8 int32 on the device that receive the status block of this call
+ *    (same slots as moe_status) once the work has run. */
+#define MOE_NOALLOC_SCRATCH_BYTES (2u << 20)
+int moe_dispatch_noalloc(const moe_shape_t* shape, const void* x, const int32_t* topk_idx,
+                         const moe_layout_t* layout, void* xg, int32_t* status_out, void* stream);
 
 /* Byte offsets of named regions inside the workspace, for tests and profilers:
  * out[0] status, out[1] h (GEMM-1 output [T*k, f] bf16), out[2] o scratch used

@@ -25,6 +25,8 @@ MOE_ERR_UNSUPPORTED_SHAPE = -2
 MOE_ERR_WORKSPACE_TOO_SMALL = -3
 MOE_ERR_MISALIGNED = -4
 MOE_ERR_CUDA = -5
+MOE_ERR_SCRATCH_LIMIT = -6
+MOE_NOALLOC_SCRATCH_BYTES = 2 << 20
 MOE_DEV_TIMEOUT = 1
 MOE_DEV_INDEX_OUT_OF_RANGE = 2
 MOE_WARN_NONFINITE_LOGIT = 1
@@ -32,7 +34,7 @@ MOE_FLAG_WEIGHT_IN_COMBINE = 1
 
 EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "moe_status", "moe_strerror",
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",
-           "moe_profile_enable", "moe_profile_read")
+           "moe_profile_enable", "moe_profile_read", "moe_dispatch_noalloc")
 
 
 class MoEShape(ctypes.Structure):
@@ -76,6 +78,7 @@ def lib() -> ctypes.CDLL:
         L.moe_combine.argtypes = [shp, vp, lay, vp, vp, vp, vp, vp, sz, vp]
         L.moe_layer.argtypes = [shp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, lay, vp, sz, vp]
         L.moe_layer_host.argtypes = [shp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.moe_dispatch_noalloc.argtypes = [shp, vp, vp, lay, vp, vp, vp]
         L.moe_profile_enable.argtypes = [ctypes.c_int]
         L.moe_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
         for name in EXPORTS:
@@ -172,6 +175,17 @@ def moe_dispatch(shape, x, topk_idx, layout: Layout, xg, ws, stream=None) -> Non
     c = layout.c()
     _check("moe_dispatch", lib().moe_dispatch(ctypes.byref(shape), _ptr(x), _ptr(topk_idx), ctypes.byref(c),
                                               _ptr(xg), _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def moe_dispatch_noalloc(shape, x, topk_idx, layout: Layout, xg, status_out=None, stream=None) -> None:
+    """moe_dispatch for callers that cannot pass a workspace (plugins inside a pre-planned memory
+    arena, allocation-free serving loops): the scratch tables live in a fixed array inside the
+    library.  Shapes beyond MOE_NOALLOC_SCRATCH_BYTES raise MoEError(MOE_ERR_SCRATCH_LIMIT).  Calls
+    on one device share that array, so keep them ordered on one stream."""
+    c = layout.c()
+    _check("moe_dispatch_noalloc", lib().moe_dispatch_noalloc(ctypes.byref(shape), _ptr(x), _ptr(topk_idx),
+                                                              ctypes.byref(c), _ptr(xg), _ptr(status_out),
+                                                              _stream(stream)))
 
 
 def moe_expert_ffn(shape, xg, layout: Layout, topk_w, w1, w3, w2, o, ws, stream=None) -> None:

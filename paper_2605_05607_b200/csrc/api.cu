@@ -224,6 +224,7 @@ const char* moe_strerror(int code) {
     case MOE_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
     case MOE_ERR_MISALIGNED: return "misaligned pointer";
     case MOE_ERR_CUDA: return "CUDA error (or no CUDA device)";
+    case MOE_ERR_SCRATCH_LIMIT: return "shape needs more scratch than the built-in no-allocation array holds";
     case MOE_DEV_TIMEOUT: return "device: bounded wait expired";
     case MOE_DEV_INDEX_OUT_OF_RANGE: return "device: expert index out of range";
     default: return "unknown code";
