@@ -28,7 +28,7 @@ from paper_2605_05607_b200 import synth  # noqa: E402
 
 METRIC = "fused MoE layer tokens/sec"
 UNIT = "tokens/s"
-KERNELS_PER_STEP = 9  # gate, topk, masks, scan, offsets, fill, gemm1, gemm2, combine
+KERNELS_PER_STEP = 10  # gate split, gate, topk, masks, scan, offsets, fill, gemm1, gemm2, combine
 
 # DRAM bytes (read + write) of one GEMM-1 launch from ncu captures summarised under profiles/;
 # None until a capture of that workload exists.
@@ -279,9 +279,8 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     # weights replicated (same seed on every rank), tokens differ per rank
-    t = synth.make_inputs(cfg, "cuda")
-    if rank > 0:
-        t["x"] = synth.make_routing_inputs(cfg.with_(seed=cfg.seed + 7919 * rank), "cuda")["x"]
+    from paper_2605_05607_b200 import replicas
+    t = replicas.make_rank_inputs(cfg, rank, "cuda")
     shape = B.make_shape(cfg)
     ws = B.alloc_workspace(shape)
     y = torch.zeros(cfg.T, cfg.d, dtype=torch.bfloat16, device="cuda")
@@ -316,10 +315,7 @@ def main():
     elapsed_ms = ev0.elapsed_time(ev1)
     g1_ms, g1_launches = B.moe_profile_read()
     B.moe_profile_enable(0)
-    if dist is not None:
-        tmax = torch.tensor([elapsed_ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tmax.item())
+    elapsed_ms = replicas.max_over_ranks(elapsed_ms, dist, "cuda")
     status = B.moe_status(ws)
     assert status[0] == 0, f"device status {status}"
 
@@ -343,10 +339,7 @@ def main():
         e1.record()
         barrier()
         e2e_ms = e0.elapsed_time(e1)
-        if dist is not None:
-            tmax = torch.tensor([e2e_ms], device="cuda")
-            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tmax.item())
+        e2e_ms = replicas.max_over_ranks(e2e_ms, dist, "cuda")
 
     clocks = None
     if sampler is not None:
@@ -368,7 +361,7 @@ def main():
 
     pk = peaks()
     tokens = cfg.T * world * args.steps
-    value = tokens / (elapsed_ms * 1e-3)
+    value = replicas.whole_job_tokens_per_s(cfg, world, args.steps, elapsed_ms)
     flops_g1 = 4.0 * cfg.P * cfg.d * cfg.f                      # GEMM-1: x W1 and x W3
     g1_avg_s = (g1_ms / max(g1_launches, 1)) * 1e-3
     achieved = flops_g1 / g1_avg_s / 1e12 if g1_launches else None

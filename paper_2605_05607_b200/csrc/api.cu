@@ -14,7 +14,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Regions of the workspace, in order.  Every region starts on a 1 KiB boundary.
 struct WsPlan {
-  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, h, o, logits, topk_idx, topk_w;
+  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, wsplit, h, o, logits, topk_idx, topk_w;
   size_t expert_counts, expert_offsets, group_counts, group_offsets, pair_row, row_pair, al, disp_token, row_src;
   size_t total;
   int W;
@@ -42,6 +42,7 @@ WsPlan plan(const moe_shape_t& s) {
   p.gprefix = take(G * W * 4);
   p.mt_prefix = take((E + 1) * 4);
   p.mp_prefix = take((E + 1) * 4);
+  p.wsplit = take(gate_split_bytes(s.d, s.E));
   p.h = take(P * (size_t)s.f * 2);
   p.o = take(P * (size_t)s.d * 2);
   p.logits = take(T * E * 4);
@@ -239,7 +240,7 @@ int moe_route(const moe_shape_t* shape, const void* x, const float* w_gate, cons
   if (logits == nullptr || topk_idx == nullptr || topk_w == nullptr) return MOE_ERR_INVALID_ARG;
   if (w_gate != nullptr && x == nullptr) return MOE_ERR_INVALID_ARG;
   if (bias_row_stride != 0 && bias_row_stride != shape->E) return MOE_ERR_INVALID_ARG;
-  if (!aligned(x, 16) || !aligned(w_gate, 16) || !aligned(logits, 16) || !aligned(topk_idx, 16) ||
+  if (!aligned(x, 128) || !aligned(w_gate, 16) || !aligned(logits, 16) || !aligned(topk_idx, 16) ||
       !aligned(topk_w, 16) || !aligned(logit_bias, 4))
     return MOE_ERR_MISALIGNED;
   WsPlan p;
@@ -247,7 +248,8 @@ int moe_route(const moe_shape_t* shape, const void* x, const float* w_gate, cons
   if (!have_device()) return MOE_ERR_CUDA;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const Shape s = to_shape(*shape);
-  if (w_gate != nullptr) TCMOE_CUDA(launch_gate_logits(s, x, w_gate, logits, st));
+  if (w_gate != nullptr)
+    TCMOE_CUDA(launch_gate_logits(s, x, w_gate, logits, at<void>(ws, p.wsplit), at<int32_t>(ws, p.status), st));
   TCMOE_CUDA(launch_topk(s, logits, logit_bias, bias_row_stride, topk_idx, topk_w, at<int32_t>(ws, p.status), st));
   return MOE_OK;
 }
@@ -355,7 +357,7 @@ int moe_layer(const moe_shape_t* shape, const void* x, const float* w_gate, cons
                at<int32_t>(ws, p.al),            at<int32_t>(ws, p.disp_token),     at<int32_t>(ws, p.row_src)};
   }
   // gate
-  TCMOE_CUDA(launch_gate_logits(s, x, w_gate, lg, st));
+  TCMOE_CUDA(launch_gate_logits(s, x, w_gate, lg, at<void>(ws, p.wsplit), status, st));
   TCMOE_CUDA(launch_topk(s, lg, logit_bias, bias_row_stride, idx, tw, status, st));
   // layout only: the dispatched copy xg is never written, GEMM-1 gathers token rows from x
   TCMOE_CUDA(launch_layout(s, idx, L, scratch(ws, p), status, st));

@@ -42,8 +42,11 @@ struct LayoutScratch {
   int W;
 };
 
+// gate_gemm.cu: wsplit is scratch of gate_split_bytes(d, E) bytes for the bf16 hi/mid/lo terms of w_gate
+size_t gate_split_bytes(int d, int E);
+cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gate, float* logits, void* wsplit,
+                               int32_t* status, cudaStream_t st);
 // route.cu
-cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gate, float* logits, cudaStream_t st);
 cudaError_t launch_topk(const Shape& s, const float* logits, const float* bias, int64_t bias_stride,
                         int32_t* topk_idx, float* topk_w, int32_t* status, cudaStream_t st);
 // layout.cu

@@ -1,106 +1,12 @@
-// Gate of the MoE layer (paper Sec. II-A: "topk experts selected by the gate network").
-//   gate_logits_kernel : logits[T,E] = x[T,d] (bf16) * w_gate[d,E] (fp32), fp32 accumulation
-//   topk_kernel        : key = logit + bias; k largest keys per token ordered by
-//                        (key descending, expert index ascending); gate weights over the k keys
+// Routing of the MoE layer (paper Sec. II-A: "topk experts selected by the gate network"); the
+// gate logits themselves are computed in gate_gemm.cu.
+//   topk_kernel : key = logit + bias; k largest keys per token ordered by
+//                 (key descending, expert index ascending); gate weights over the k keys
 #include "common.cuh"
 
 #include <cuda_bf16.h>
 
 namespace tcmoe {
-
-// ------------------------------------------------------------------------------------------------
-// Gate logits: register-tiled fp32 GEMM.  256 threads; thread grid (256 / (BN/4)) x (BN/4);
-// each thread owns TM x 4 outputs.  x tile is converted to fp32 and stored k-major in shared
-// memory so that the inner product reads are conflict-free broadcasts.
-// ------------------------------------------------------------------------------------------------
-template <int BN>
-struct GateCfg {
-  static constexpr int TN = 4;
-  static constexpr int TX = BN / TN;          // threads along experts
-  static constexpr int TY = 256 / TX;         // threads along tokens
-  static constexpr int BM = (BN >= 64) ? 64 : (BN >= 32 ? 64 : 128);
-  static constexpr int TM = BM / TY;
-  static constexpr int BK = 32;
-};
-
-template <int BN>
-__global__ void __launch_bounds__(256) gate_logits_kernel(const __nv_bfloat16* __restrict__ x,
-                                                          const float* __restrict__ wg,
-                                                          float* __restrict__ logits, int T, int d, int E) {
-  using C = GateCfg<BN>;
-  constexpr int BM = C::BM, BK = C::BK, TM = C::TM, TN = C::TN;
-  __shared__ float xs[BK][BM + 4];
-  __shared__ float ws[BK][BN];
-  const int tid = threadIdx.x;
-  const int tx = tid % C::TX, ty = tid / C::TX;
-  const int m0 = blockIdx.x * BM, n0 = blockIdx.y * BN;
-  float acc[TM][TN];
-#pragma unroll
-  for (int i = 0; i < TM; ++i)
-#pragma unroll
-    for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
-
-  for (int k0 = 0; k0 < d; k0 += BK) {
-    // x tile: BM rows x BK cols, 16-byte vectors of 8 bf16 (d % 8 == 0)
-    for (int v = tid; v < BM * (BK / 8); v += 256) {
-      const int r = v / (BK / 8), c = (v % (BK / 8)) * 8;
-      const int row = m0 + r, col = k0 + c;
-      uint4 raw = make_uint4(0, 0, 0, 0);
-      if (row < T && col < d) raw = __ldg(reinterpret_cast<const uint4*>(x + (size_t)row * d + col));
-      const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const float2 f2 = __bfloat1622float2(p[q]);
-        xs[c + 2 * q][r] = f2.x;
-        xs[c + 2 * q + 1][r] = f2.y;
-      }
-    }
-    for (int v = tid; v < BK * BN; v += 256) {
-      const int kk = v / BN, nn = v % BN;
-      const int row = k0 + kk, col = n0 + nn;
-      ws[kk][nn] = (row < d && col < E) ? __ldg(wg + (size_t)row * E + col) : 0.f;
-    }
-    __syncthreads();
-#pragma unroll 8
-    for (int kk = 0; kk < BK; ++kk) {
-      float a[TM], b[TN];
-#pragma unroll
-      for (int i = 0; i < TM; ++i) a[i] = xs[kk][ty * TM + i];
-#pragma unroll
-      for (int j = 0; j < TN; ++j) b[j] = ws[kk][tx * TN + j];
-#pragma unroll
-      for (int i = 0; i < TM; ++i)
-#pragma unroll
-        for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
-    }
-    __syncthreads();
-  }
-#pragma unroll
-  for (int i = 0; i < TM; ++i) {
-    const int row = m0 + ty * TM + i;
-    if (row >= T) continue;
-#pragma unroll
-    for (int j = 0; j < TN; ++j) {
-      const int col = n0 + tx * TN + j;
-      if (col < E) logits[(size_t)row * E + col] = acc[i][j];
-    }
-  }
-}
-
-template <int BN>
-static cudaError_t launch_gate_bn(const Shape& s, const void* x, const float* wg, float* logits, cudaStream_t st) {
-  dim3 grid((s.T + GateCfg<BN>::BM - 1) / GateCfg<BN>::BM, (s.E + BN - 1) / BN);
-  ProfileScope prof(KID_GATE, st);
-  gate_logits_kernel<BN><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(x), wg, logits, s.T, s.d, s.E);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gate, float* logits, cudaStream_t st) {
-  if (s.T == 0) return cudaSuccess;
-  if (s.E <= 8) return launch_gate_bn<8>(s, x, w_gate, logits, st);
-  if (s.E <= 32) return launch_gate_bn<32>(s, x, w_gate, logits, st);
-  return launch_gate_bn<64>(s, x, w_gate, logits, st);
-}
 
 // ------------------------------------------------------------------------------------------------
 // Top-k: one warp per token.  Lane l holds experts l, l+32, ... (KPL of them) as order-preserving
