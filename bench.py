@@ -32,7 +32,7 @@ KERNELS_PER_STEP = 10  # gate split, gate, topk, masks, scan, offsets, fill, gem
 
 # DRAM bytes (read + write) of one GEMM-1 launch from ncu captures summarised under profiles/;
 # None until a capture of that workload exists.
-GEMM1_DRAM_TRAFFIC = {}
+GEMM1_DRAM_TRAFFIC = {"C2": 1.944110e9 + 228.062e6}   # profiles/ffn_gemm_C2_ncu_full.md
 
 
 def peaks():
@@ -148,7 +148,7 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
-def stage_breakdown(cfg, t, reps=5):
+def stage_breakdown(cfg, t, reps=5, with_ffn=True):
     """Per-stage device times of the unfused entry points and of the fused layer, cold L2
     (a 512 MB buffer is overwritten before every timed call), with algorithmic bytes / flops."""
     from paper_2605_05607_b200 import binding as B
@@ -165,6 +165,8 @@ def stage_breakdown(cfg, t, reps=5):
     y = torch.zeros(T, d, dtype=torch.bfloat16, device=dev)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
 
+    if not with_ffn:
+        o.copy_(torch.randn(o.shape, device=dev, dtype=torch.float32).to(torch.bfloat16))
     calls = {
         "route": lambda: B.moe_route(shape, t["x"], t["w_gate"], t["bias"], logits, idx, w, ws),
         "layout": lambda: B.moe_dispatch(shape, t["x"], idx, lay, None, ws),
@@ -175,6 +177,8 @@ def stage_breakdown(cfg, t, reps=5):
     }
     kernels = {"route": ["gate", "topk"], "dispatch": ["dispatch"], "expert_ffn": ["gemm1", "gemm2"],
                "combine": ["combine"]}
+    if not with_ffn:
+        del calls["expert_ffn"], calls["layer_fused"]
     out = {}
     for name, fn in calls.items():
         fn()                                           # warm (and produces the next stage's input)
@@ -201,6 +205,17 @@ def stage_breakdown(cfg, t, reps=5):
     comb_bytes = (P + T) * 2.0 * d + 12.0 * P
     flops = 6.0 * P * d * f
     dk, ck = out["dispatch"]["dispatch_kernel_ms"], out["combine"]["combine_kernel_ms"]
+    gate_ms = out["route"]["gate_kernel_ms"]
+    out["route"].update(gate_flops_bf16=6.0 * T * d * E, gate_tflops_bf16=6.0 * T * d * E / gate_ms / 1e9,
+                        gate_x_gbs=2.0 * T * d / gate_ms / 1e6)
+    if not with_ffn:
+        out["dispatch"].update(bytes=disp_bytes, gbs=disp_bytes / dk / 1e6,
+                               frac_hbm_measured=disp_bytes / dk / 1e6 / pk["hbm_gbs"])
+        out["combine"].update(bytes=comb_bytes, gbs=comb_bytes / ck / 1e6,
+                              frac_hbm_measured=comb_bytes / ck / 1e6 / pk["hbm_gbs"])
+        out["summary"] = {"n_disp": n_disp, "pairs": P, "dedup": 1.0 - n_disp / P,
+                          "timing": "cold L2 (512 MB overwrite before each call)"}
+        return out
     g1, g2 = out["expert_ffn"]["gemm1_kernel_ms"], out["expert_ffn"]["gemm2_kernel_ms"]
     out["dispatch"].update(bytes=disp_bytes, gbs=disp_bytes / dk / 1e6, frac_hbm_measured=disp_bytes / dk / 1e6 / pk["hbm_gbs"])
     out["combine"].update(bytes=comb_bytes, gbs=comb_bytes / ck / 1e6, frac_hbm_measured=comb_bytes / ck / 1e6 / pk["hbm_gbs"])
@@ -251,17 +266,27 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="C2", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--shape", default=None, metavar="T,d,f,E,k,G",
+                    help="override the sizes of --config (keeps its score function and router bias); "
+                         "for profiler captures of a slice that fits the capture size rules")
     ap.add_argument("--impl", default="tcmoe", choices=["tcmoe", "reference"])
     ap.add_argument("--ref-sample", type=int, default=0,
                     help="tokens per step of the reference arm (0: sized from a one-token calibration)")
     ap.add_argument("--cpu-sample", type=int, default=64, help="tokens of the cpu_baseline leg (0: skip)")
     ap.add_argument("--lean", action="store_true",
                     help="timed region only: no e2e / stage / cpu_baseline legs (for profiler captures)")
+    ap.add_argument("--stages-only", action="store_true",
+                    help="only the per-stage breakdown of --config (prints its JSON); for profiler captures")
+    ap.add_argument("--no-ffn", action="store_true", help="with --stages-only: skip expert weights and the FFN")
+    ap.add_argument("--reps", type=int, default=5, help="timed repetitions per stage in the breakdown")
     ap.add_argument("--report", default=None,
                     help="also write per-stage numbers of every configuration to this JSON file (1 GPU)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "tcmoe" else args.warmup
     cfg = synth.CONFIGS[args.config]
+    if args.shape:
+        T, d, f, E, k, G = (int(v) for v in args.shape.split(","))
+        cfg = cfg.with_(name=f"{cfg.name}-slice", T=T, d=d, f=f, E=E, k=k, G=G)
 
     if args.impl == "reference":
         run_reference(args, cfg)
@@ -269,6 +294,11 @@ def main():
 
     from paper_2605_05607_b200 import binding as B
     B.lib()  # fail loudly if the CUDA library is missing
+    if args.stages_only:
+        torch.cuda.set_device(0)
+        t = synth.make_routing_inputs(cfg, "cuda") if args.no_ffn else synth.make_inputs(cfg, "cuda")
+        print(json.dumps({"config": cfg.name, "stages": stage_breakdown(cfg, t, args.reps, not args.no_ffn)}), flush=True)
+        return
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

@@ -23,6 +23,11 @@ SMALL = [
     synth.MoEConfig("G=E-local", T=200, d=256, f=128, E=16, k=4, G=16, bias="locality", boost=2.0, seed=5),
     synth.MoEConfig("one-expert", T=300, d=192, f=448, E=1, k=1, G=1, seed=6),
     synth.MoEConfig("gptoss-ish", T=512, d=2880 // 5, f=2880 // 5, E=32, k=4, G=8, bias="zipf", zipf_s=1.1, seed=7),
+    # more experts than one 256-column gate tile, experts per lane > 8 in top-k, sigmoid scores
+    synth.MoEConfig("E320", T=260, d=136, f=72, E=320, k=6, G=10, score_fn=1, seed=8),
+    # a single token; many tokens in a single expert pair tile boundary (257 rows: 128 + 128 + 1)
+    synth.MoEConfig("T1", T=1, d=64, f=64, E=8, k=2, G=2, seed=9),
+    synth.MoEConfig("rows257", T=257, d=64, f=192, E=2, k=2, G=1, seed=10),
 ]
 
 
@@ -171,4 +176,14 @@ def test_degenerate_and_error_paths():
     st = run.status()
     assert st[0] == B.MOE_DEV_INDEX_OUT_OF_RANGE and st[3] == 99
     B.moe_status_reset(run.ws)
+    assert run.status()[0] == 0
+
+
+def test_route_limits_E1024_k32():
+    cfg = synth.MoEConfig("E1024", T=130, d=72, f=64, E=1024, k=32, G=8, bias="zipf", zipf_s=0.7, seed=12)
+    run = H.Run(cfg, inputs=synth.make_routing_inputs(cfg, "cuda") | {"w1": None, "w3": None, "w2": None})
+    run.route()
+    idx_ref, _ = H.check_route(run)
+    run.dispatch()
+    H.check_layout(run, idx_ref)
     assert run.status()[0] == 0
