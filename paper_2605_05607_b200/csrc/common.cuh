@@ -74,6 +74,8 @@ struct FfnArgs {
 };
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st);
 int sm_count();
+int current_device();   // index of the current CUDA device, clamped to [0, MAX_DEVICES)
+constexpr int MAX_DEVICES = 64;   // per-device caches (kernel attributes, SM counts) are arrays of this size
 
 // Optional event bracket around launches of one kernel id (see moe_profile_enable).
 struct ProfileScope {

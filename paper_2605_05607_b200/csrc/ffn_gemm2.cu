@@ -213,7 +213,8 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
 
 // Persistent grid: two CTAs per resident cluster, at most one CTA per SM.
 int pair_grid() {
-  static int g = 0;
+  static int grid_of[MAX_DEVICES] = {};
+  int& g = grid_of[current_device()];
   if (g == 0) {
     int clusters = 0;
     cudaLaunchConfig_t cfg = {};
@@ -239,11 +240,12 @@ int pair_grid() {
 }  // namespace
 
 cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[MAX_DEVICES] = {};   // the attribute is per device
+  const int dev = current_device();
+  if (!attr_set[dev]) {
     cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[dev] = true;
   }
   ProfileScope prof(KID_GEMM2, st);
   ffn_gemm2_kernel<<<pair_grid(), THREADS, SMEM_BYTES, st>>>(m_w2, m_h, p);

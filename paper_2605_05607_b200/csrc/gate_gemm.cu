@@ -198,11 +198,12 @@ size_t gate_split_bytes(int d, int E) { return (size_t)3 * d * ((E + 63) & ~63) 
 cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gate, float* logits, void* wsplit,
                                int32_t* status, cudaStream_t st) {
   if (s.T == 0) return cudaSuccess;
-  static bool attr_set = false;
-  if (!attr_set) {
+  static bool attr_set[MAX_DEVICES] = {};   // the attribute is per device
+  const int dev = current_device();
+  if (!attr_set[dev]) {
     cudaError_t e = cudaFuncSetAttribute(gate_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set[dev] = true;
   }
   const int Epad = (s.E + 63) & ~63;
   EncodeTiledFn fn = encoder();
