@@ -8,7 +8,13 @@
 // (120 GFLOP, 3.7 ms for the DeepSeek-V3-shaped layer); the tensor pipe does 3x that in ~0.3 ms.
 //
 // One CTA per (128-token tile, 256-expert tile); warps 0-3 epilogue (TMEM -> fp32 stores), warp 4
-// TMA producer, warp 5 UMMA issuer and TMEM owner; 4 stages of (A 16 KB + B up to 32 KB).
+// TMA producer, warp 5 UMMA issuer and TMEM owner.  Two schedules:
+//  - E <= 128 ("side by side"): the hi / mid / lo slabs of a k-block sit next to each other as
+//    columns of one B tile (3 x ceil(E/64) slabs <= 6), x is loaded once per k-block, one or two
+//    UMMAs fill separate accumulator column groups and the epilogue adds the three groups;
+//    d/64 iterations of (A 16 KB + B <= 48 KB), 3 stages.
+//  - larger E: the three terms are accumulated in place, 3 d/64 iterations of (A 16 KB + B 32 KB),
+//    4 stages (the accumulators of 3 x 256 columns would not fit the 512 TMEM columns).
 #include "ffn_common.cuh"
 
 namespace tcmoe {
@@ -16,12 +22,11 @@ namespace {
 
 using namespace ffn;
 
-constexpr int NSTAGE = 4;
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int B_BYTES_MAX = UMMA_N * BK * 2;
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES_MAX;
-constexpr int NUM_BARS = 2 * NSTAGE + 1;
-constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64;
+constexpr int MAX_STAGES = 4;
+constexpr int NUM_BARS = 2 * MAX_STAGES + 1;
+constexpr int RING_BYTES = 4 * (A_BYTES + 4 * 8192);   // = 3 * (A_BYTES + 6 * 8192) = 192 KiB
+constexpr int SMEM_BYTES = 1024 + RING_BYTES + NUM_BARS * 8 + 64;
 constexpr int THREADS = 192;
 
 // w_gate fp32 [d, E] -> bf16 [3, d, Epad]: hi, mid, lo terms, zero in the padding columns
@@ -44,6 +49,7 @@ __global__ void __launch_bounds__(256) split_gate_kernel(const float* __restrict
 struct GateParams {
   float* logits;
   int T, E, KB, n_tiles;
+  int side_by_side;   // 1: hi | mid | lo as column groups of one B tile (E <= 128)
   int32_t* status;
 };
 
@@ -52,26 +58,30 @@ gate_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
                  const GateParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + NSTAGE * STAGE_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + RING_BYTES);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
   int* abort_s = reinterpret_cast<int*>(tmem_slot + 1);
 
   const uint32_t smem_base = ptx::smem_u32(smem);
   const uint32_t bar_base = ptx::smem_u32(bars);
   auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (NSTAGE + s); };
-  const uint32_t done_bar = bar_base + 8u * (2 * NSTAGE);
+  auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
+  const uint32_t done_bar = bar_base + 8u * (2 * MAX_STAGES);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int mt = blockIdx.x / p.n_tiles, nt = blockIdx.x % p.n_tiles;
   const int row0 = mt * BM, n0 = nt * UMMA_N;
   const int ncols = min(UMMA_N, ((p.E - n0) + 63) & ~63);   // expert columns of this tile, in 64-column slabs
   const int nslab = ncols >> 6;
-  const int iters = 3 * p.KB;
+  const bool sbs = p.side_by_side != 0;
+  const int bslabs = sbs ? 3 * nslab : nslab;            // B slabs per stage
+  const int NSTAGE = sbs ? 3 : 4;
+  const int STAGE_BYTES = A_BYTES + (sbs ? 6 : 4) * 8192;
+  const int iters = sbs ? p.KB : 3 * p.KB;
 
   if (threadIdx.x == 0) {
     *abort_s = p.status[ST_ABORT];
-    for (int s = 0; s < NSTAGE; ++s) {
+    for (int s = 0; s < MAX_STAGES; ++s) {
       ptx::mbar_init(full_bar(s), 1);
       ptx::mbar_init(empty_bar(s), 1);
     }
@@ -83,7 +93,7 @@ gate_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     ptx::prefetch_tensormap(&map_w);
   }
   if (warp == 5) {
-    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 256);
+    ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
     ptx::tmem_relinquish();
   }
   ptx::tc_fence_before();
@@ -113,6 +123,16 @@ gate_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
         for (int c = 0; c < ncols; c += 32) {
           uint32_t acc[32];
           ptx::tmem_ld32(taddr + c, acc);
+          if (sbs) {   // logits = (hi + mid) + lo: the three column groups are ncols apart
+            uint32_t mid[32], lo[32];
+            ptx::tmem_ld32(taddr + ncols + c, mid);
+            ptx::tmem_ld32(taddr + 2 * ncols + c, lo);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int v = 0; v < 32; ++v)
+              acc[v] = __float_as_uint(__fadd_rn(__fadd_rn(__uint_as_float(acc[v]), __uint_as_float(mid[v])),
+                                                 __uint_as_float(lo[v])));
+          }
           ptx::tmem_ld_wait();
           if (valid) {
             if (vec) {
@@ -134,14 +154,23 @@ gate_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   } else if (warp == 4) {
     // ================================ TMA producer ================================
     if (lane == 0 && !*abort_flag) {
+      int slab_col[6], slab_split[6];   // slab c = (split c / nslab, 64-column slab c % nslab), hoisted out of the loop
+#pragma unroll
+      for (int c = 0; c < 6; ++c) {
+        slab_col[c] = n0 + (c % nslab) * 64;
+        slab_split[c] = c / nslab;
+      }
+      int s = 0, ph = 1;
       for (int it = 0; it < iters; ++it) {
-        const int s = it % NSTAGE;
-        if (!ptx::mbar_wait(empty_bar(s), ((it / NSTAGE) & 1) ^ 1, abort_flag, global_abort)) { timeout(2); break; }
+        if (!ptx::mbar_wait(empty_bar(s), ph, abort_flag, global_abort)) { timeout(2); break; }
         const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
-        const int kb = it / 3, split = it - kb * 3;
-        ptx::mbar_arrive_expect_tx(full_bar(s), A_BYTES + nslab * 8192);
+        const int kb = sbs ? it : it / 3, split0 = sbs ? 0 : it - kb * 3;
+        ptx::mbar_arrive_expect_tx(full_bar(s), A_BYTES + bslabs * 8192);
         ptx::tma_load_2d(sa, &map_x, full_bar(s), kb * BK, row0);
-        for (int c = 0; c < nslab; ++c) ptx::tma_load_3d(sb + c * 8192, &map_w, full_bar(s), n0 + c * 64, kb * BK, split);
+#pragma unroll
+        for (int c = 0; c < 6; ++c)
+          if (c < bslabs) ptx::tma_load_3d(sb + c * 8192, &map_w, full_bar(s), slab_col[c], kb * BK, split0 + slab_split[c]);
+        if (++s == NSTAGE) { s = 0; ph ^= 1; }
       }
     }
   } else {
@@ -149,19 +178,26 @@ gate_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     if (lane == 0 && !*abort_flag) {
       const uint64_t a_base = desc_base(16, 1024);
       const uint64_t b_base = desc_base(BK * 128, 1024);
-      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(ncols >> 3) << 17) |
-                             ((uint32_t)(BM >> 4) << 24);
+      auto idesc_n = [](int n) {
+        return (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      };
+      const int n_first = min(bslabs, 4) * 64, n_second = (bslabs - min(bslabs, 4)) * 64;   // columns per UMMA
       bool ok = true;
+      int s = 0, ph = 0;
       for (int it = 0; it < iters; ++it) {
-        const int s = it % NSTAGE;
-        if (!ptx::mbar_wait(full_bar(s), (it / NSTAGE) & 1, abort_flag, global_abort)) { timeout(3); ok = false; break; }
+        if (!ptx::mbar_wait(full_bar(s), ph, abort_flag, global_abort)) { timeout(3); ok = false; break; }
         ptx::tc_fence_after();
         const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
         const uint64_t ad = desc_at(a_base, sa), bd = desc_at(b_base, sb);
 #pragma unroll
-        for (int k = 0; k < BK / 16; ++k)
-          ptx::umma_bf16(tmem_base, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), idesc, (it | k) != 0);
+        for (int k = 0; k < BK / 16; ++k) {
+          ptx::umma_bf16(tmem_base, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), idesc_n(n_first), (it | k) != 0);
+          if (n_second > 0)   // slabs 4, 5 start 4 * 8 KiB into the B tile and 256 columns into the accumulator
+            ptx::umma_bf16(tmem_base + 256, ad + (uint64_t)(k * 2), bd + (uint64_t)(2048 + k * 128), idesc_n(n_second),
+                           (it | k) != 0);
+        }
         ptx::umma_commit(empty_bar(s));
+        if (++s == NSTAGE) { s = 0; ph ^= 1; }
       }
       if (ok) ptx::umma_commit(done_bar);
     }
@@ -175,7 +211,7 @@ gate_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   __syncthreads();
   if (warp == 5) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, 256);
+    ptx::tmem_dealloc(tmem_base, 512);
   }
 }
 
@@ -240,6 +276,7 @@ cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gat
   p.E = s.E;
   p.KB = (s.d + BK - 1) / BK;
   p.n_tiles = (s.E + UMMA_N - 1) / UMMA_N;
+  p.side_by_side = s.E <= 128 ? 1 : 0;
   p.status = status;
   const int grid = ((s.T + BM - 1) / BM) * p.n_tiles;
   gate_umma_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(m_x, m_w, p);
