@@ -35,9 +35,15 @@ struct Tile {
   int e, n0, row0, rows;
 };
 
-// Task w -> (expert, n-tile, m-tile), ordered expert-major, then n-tile, m-tile fastest so that
-// CTAs running at the same time share the weight tile in L2.  `rows_per_tile` is 128 (one CTA) or
-// 256 (a CTA pair; CTA `rank` owns the rank-th half).  rows <= 0: nothing of this CTA is valid.
+// Task w -> (expert, m-group, n-tile, m-tile in group): expert-major; inside an expert the m-tiles
+// are taken in groups of M_GROUP, and inside a group the order is n-tile, m-tile fastest.  CTAs
+// that run at the same time then share the weight tile (same expert, same n) in L2, and the
+// activation rows that must stay in L2 while the n-tiles sweep over them are bounded by one
+// m-group (a popular expert with hundreds of m-tiles would otherwise cycle all of its rows through
+// L2 once per n-tile).  `rows_per_tile` is 128 (one CTA) or 256 (a CTA pair; CTA `rank` owns the
+// rank-th half).  rows <= 0: nothing of this CTA is valid.
+constexpr int M_GROUP_ROWS = 2048;   // rows of one m-group
+
 __device__ __forceinline__ Tile decode_tile(int w, const int* tp, const int* eoff, int E, int n_tiles, int bn_out,
                                             int rows_per_tile, int rank) {
   int lo = 0, hi = E;  // tp[lo] * n_tiles <= w < tp[hi] * n_tiles
@@ -45,12 +51,16 @@ __device__ __forceinline__ Tile decode_tile(int w, const int* tp, const int* eof
     const int mid = (lo + hi) >> 1;
     if (tp[mid] * n_tiles <= w) lo = mid; else hi = mid;
   }
-  const int local = w - tp[lo] * n_tiles;
+  int local = w - tp[lo] * n_tiles;
   const int mt = tp[lo + 1] - tp[lo];
+  const int mg = M_GROUP_ROWS / rows_per_tile;          // m-tiles per full group
+  const int g = local / (mg * n_tiles);                 // group index
+  local -= g * mg * n_tiles;
+  const int gsize = min(mg, mt - g * mg);               // m-tiles in this group
   Tile t;
   t.e = lo;
-  t.n0 = (local / mt) * bn_out;
-  t.row0 = eoff[lo] + (local % mt) * rows_per_tile + rank * BM;
+  t.n0 = (local / gsize) * bn_out;
+  t.row0 = eoff[lo] + (g * mg + local % gsize) * rows_per_tile + rank * BM;
   t.rows = min(BM, eoff[lo + 1] - t.row0);
   return t;
 }
