@@ -263,8 +263,9 @@ def workload_config(cfg, n_gpus):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps (default 200: ~0.5 s on C2, long enough for clock samples; reference arm: 8)")
+    ap.add_argument("--warmup", type=int, default=None, help="untimed warm-up steps (default 10; reference arm: 2)")
     ap.add_argument("--config", default="C2", choices=sorted(synth.CONFIGS))
     ap.add_argument("--shape", default=None, metavar="T,d,f,E,k,G",
                     help="override the sizes of --config (keeps its score function and router bias); "
@@ -282,6 +283,10 @@ def main():
     ap.add_argument("--report", default=None,
                     help="also write per-stage numbers of every configuration to this JSON file (1 GPU)")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 200 if args.impl == "tcmoe" else 8
+    if args.warmup is None:
+        args.warmup = 10 if args.impl == "tcmoe" else 2
     args.warmup = max(args.warmup, 3) if args.impl == "tcmoe" else args.warmup
     cfg = synth.CONFIGS[args.config]
     if args.shape:
@@ -405,7 +410,7 @@ def main():
                {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.T * cfg.d * 2,
                 "d2h_bytes_per_step": cfg.T * cfg.d * 2},
         "gpu_launches": KERNELS_PER_STEP * args.steps,
-        "roofline": {"kernel": "ffn_gemm_kernel<0> (GEMM-1 + SwiGLU, tcgen05)", "bound": "tensor",
+        "roofline": {"kernel": "ffn_gemm1_kernel (GEMM-1 + SwiGLU, tcgen05)", "bound": "tensor",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": (achieved / peak) if achieved else None,
                      "peak_source": f"{pk['source']} bf16 sustained (kernel timed inside a long step)",
