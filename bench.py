@@ -150,7 +150,11 @@ def run_reference(args, cfg):
 
 def stage_breakdown(cfg, t, reps=5, with_ffn=True):
     """Per-stage device times of the unfused entry points and of the fused layer, cold L2
-    (a 512 MB buffer is overwritten before every timed call), with algorithmic bytes / flops."""
+    (a 512 MB buffer is overwritten before every timed call), with algorithmic bytes / flops.
+    Stage and kernel times are ISOLATED: the device idles 0.2 s before each one, so a memory-bound
+    kernel is not timed in the low-clock state the power cap leaves behind a GEMM (measured: a plain
+    copy drops from 6.6 to 5.7 TB/s, combine from 5.7 to 4.1 TB/s right after the FFN).  The
+    in-layer times of the same kernels are reported under layer_fused (`*_kernel_ms`)."""
     from paper_2605_05607_b200 import binding as B
     shape = B.make_shape(cfg)
     ws = B.alloc_workspace(shape)
@@ -176,7 +180,7 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
         "layer_fused": lambda: B.moe_layer(shape, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws),
     }
     kernels = {"route": ["gate", "topk"], "dispatch": ["dispatch"], "expert_ffn": ["gemm1", "gemm2"],
-               "combine": ["combine"]}
+               "combine": ["combine"], "layer_fused": ["gate", "topk", "gemm1", "gemm2", "combine"]}
     if not with_ffn:
         del calls["expert_ffn"], calls["layer_fused"]
     out = {}
@@ -184,6 +188,8 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
         fn()                                           # warm (and produces the next stage's input)
         times = []
         for _ in range(reps):
+            torch.cuda.synchronize()
+            time.sleep(0.2)
             flush.fill_(1)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(); fn(); e1.record()
@@ -193,6 +199,8 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
         for kn in kernels.get(name, []):
             B.moe_profile_enable(B.KERNEL_IDS[kn])
             for _ in range(reps):
+                torch.cuda.synchronize()
+                time.sleep(0.2)
                 flush.fill_(1)
                 fn()
             ms, n = B.moe_profile_read()
@@ -242,6 +250,15 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
     for _ in range(reps):
         seq_ms.append(timed(unfused_seq))
         fus_ms.append(timed(calls["layer_fused"]))
+    # in-layer (back to back, no idle gap) kernel times of the fused call
+    for kn in kernels["layer_fused"]:
+        B.moe_profile_enable(B.KERNEL_IDS[kn])
+        for _ in range(reps):
+            calls["layer_fused"]()
+        ms, n = B.moe_profile_read()
+        B.moe_profile_enable(0)
+        out["layer_fused"][kn + "_in_layer_ms"] = ms / max(n, 1)
+    out["combine"]["in_layer_gbs"] = comb_bytes / out["layer_fused"]["combine_in_layer_ms"] / 1e6
     out["summary"] = {"unfused_sum_ms": unfused, "unfused_back_to_back_ms": float(np.median(seq_ms)),
                       "fused_back_to_back_ms": float(np.median(fus_ms)), "fused_ms": out["layer_fused"]["ms"],
                       "fused_tokens_per_s": T / out["layer_fused"]["ms"] * 1e3,
@@ -354,27 +371,54 @@ def main():
     status = B.moe_status(ws)
     assert status[0] == 0, f"device status {status}"
 
-    e2e_ms = None
+    e2e_ms = two_stream_ms = None
     if not args.lean:
-        # ---- end to end through the host-buffer entry point: pinned x in, y out, every step
+        # ---- end to end through the host-buffer entry point: every step copies its x from pinned
+        # host memory and reads its y back.  Two streams with their own staging buffers and
+        # workspaces alternate between steps, so the copies of one step overlap the kernels of the
+        # neighbouring steps (what a serving loop does); all copies stay inside the timed region.
         x_host = t["x"].cpu().pin_memory()
-        y_host = torch.empty_like(x_host).pin_memory()
-        x_dev = torch.empty_like(t["x"])
+        lanes = []
+        for _ in range(2):
+            lanes.append({"stream": torch.cuda.Stream(), "x_dev": torch.empty_like(t["x"]),
+                          "y_dev": torch.empty_like(y), "y_host": torch.empty_like(x_host).pin_memory(),
+                          "ws": B.alloc_workspace(shape)})
 
-        def step_host():
-            B.moe_layer_host(shape, x_host, x_dev, t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, y_host, ws)
+        def step_host(i):
+            ln = lanes[i & 1]
+            B.moe_layer_host(shape, x_host, ln["x_dev"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"],
+                             ln["y_dev"], ln["y_host"], ln["ws"], stream=ln["stream"])
 
-        for _ in range(3):
-            step_host()
-        barrier()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(args.steps):
-            step_host()
-        e1.record()
-        barrier()
-        e2e_ms = e0.elapsed_time(e1)
-        e2e_ms = replicas.max_over_ranks(e2e_ms, dist, "cuda")
+        def step_dev(i):   # same two-stream schedule without the copies, for comparison
+            ln = lanes[i & 1]
+            B.moe_layer(shape, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], ln["y_dev"], ln["ws"],
+                        stream=ln["stream"])
+
+        main = torch.cuda.current_stream()
+
+        def timed_two_streams(fn):
+            for i in range(4):
+                fn(i)
+            barrier()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(main)
+            for ln in lanes:
+                ln["stream"].wait_event(e0)
+            for i in range(args.steps):
+                fn(i)
+            for ln in lanes:
+                main.wait_stream(ln["stream"])
+            e1.record(main)
+            barrier()
+            return replicas.max_over_ranks(e0.elapsed_time(e1), dist, "cuda")
+
+        two_stream_ms = timed_two_streams(step_dev)
+        e2e_ms = timed_two_streams(step_host)
+        for ln in lanes:
+            st = B.moe_status(ln["ws"], stream=ln["stream"])
+            assert st[0] == 0, f"device status {st}"
+        assert torch.equal(lanes[0]["y_host"], lanes[1]["y_host"])   # same tokens in, same result out
+        del lanes
 
     clocks = None
     if sampler is not None:
@@ -408,7 +452,9 @@ def main():
         "clocks": clocks,
         "e2e": None if e2e_ms is None else
                {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.T * cfg.d * 2,
-                "d2h_bytes_per_step": cfg.T * cfg.d * 2},
+                "d2h_bytes_per_step": cfg.T * cfg.d * 2,
+                "pipeline": "moe_layer_host on 2 alternating streams (double-buffered staging and workspace)"},
+        "value_two_streams": None if two_stream_ms is None else tokens / (two_stream_ms * 1e-3),
         "gpu_launches": KERNELS_PER_STEP * args.steps,
         "roofline": {"kernel": "ffn_gemm1_kernel (GEMM-1 + SwiGLU, tcgen05)", "bound": "tensor",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
