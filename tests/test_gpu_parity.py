@@ -187,3 +187,23 @@ def test_route_limits_E1024_k32():
     run.dispatch()
     H.check_layout(run, idx_ref)
     assert run.status()[0] == 0
+
+
+def test_random_shape_sweep():
+    """Seeded sweep over small random shapes: ragged T, K and N tails (any multiple of 8), every
+    k / G / E combination the limits allow, both score functions, both weight placements."""
+    rng = np.random.default_rng(2024)
+    for i in range(14):
+        E = int(rng.choice([1, 2, 3, 4, 6, 8, 12, 16, 24, 48]))
+        G = int(rng.choice([g for g in range(1, E + 1) if E % g == 0]))
+        k = int(rng.integers(1, min(E, 6) + 1))
+        cfg = synth.MoEConfig(f"sweep{i}", T=int(rng.integers(1, 420)), d=8 * int(rng.integers(1, 40)),
+                              f=8 * int(rng.integers(1, 40)), E=E, k=k, G=G, score_fn=int(rng.integers(0, 2)),
+                              bias=str(rng.choice(["none", "zipf", "locality"])), zipf_s=1.0, boost=1.5, seed=100 + i)
+        flags = B.MOE_FLAG_WEIGHT_IN_COMBINE if i % 3 == 0 else 0
+        run, y_staged, y_def = staged(cfg, flags)
+        y2 = torch.zeros_like(run.y)
+        run.layer(y=y2)
+        y_fused = O.bf16_to_f64(H.bf16_host(y2)[: cfg.T])
+        H.assert_close_out(y_fused, y_def, f"{cfg} fused")
+        assert np.array_equal(y_fused, y_staged), cfg
