@@ -33,6 +33,7 @@ constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + 2 *
 constexpr int THREADS = 192;
 constexpr int BN_OUT = 256;
 constexpr uint32_t IDESC = idesc_bf16(2 * BM);
+constexpr uint32_t HINT = 4000;   // try_wait suspend-time hint (ns), see ptx::mbar_try_wait
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_h,
@@ -103,7 +104,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
     for (int w = cluster_id; w < total && !*abort_flag; w += num_clusters, ++tl) {
       const Tile t = tile_of(w);
       const int buf = tl & 1;
-      if (!ptx::mbar_wait_warp<true>(tfull_bar(buf), (tl >> 1) & 1, abort_flag, global_abort)) { timeout(1); break; }
+      if (!ptx::mbar_wait_warp<false, HINT>(tfull_bar(buf), (tl >> 1) & 1, abort_flag, global_abort)) { timeout(1); break; }
       ptx::tc_fence_after();
       const int lrow = warp * 32 + lane;
       const bool valid = lrow < t.rows;
@@ -146,7 +147,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
         bool ok = true;
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const int s = it % NSTAGE;
-          if (!ptx::mbar_wait(empty_bar(s), ((it / NSTAGE) & 1) ^ 1, abort_flag, global_abort)) {
+          if (!ptx::mbar_wait<false, HINT>(empty_bar(s), ((it / NSTAGE) & 1) ^ 1, abort_flag, global_abort)) {
             timeout(2); ok = false; break;
           }
           const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
@@ -170,7 +171,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
       int tl = 0;
       for (int w = cluster_id; w < total && !*abort_flag; w += num_clusters, ++tl) {
         const int buf = tl & 1;
-        if (!ptx::mbar_wait_cluster(tempty_bar(buf), ((tl >> 1) & 1) ^ 1, abort_flag, global_abort)) {
+        if (!ptx::mbar_wait_cluster<HINT>(tempty_bar(buf), ((tl >> 1) & 1) ^ 1, abort_flag, global_abort)) {
           timeout(3); break;
         }
         ptx::tc_fence_after();
@@ -178,7 +179,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
         bool ok = true;
         for (int kb = 0; kb < KB; ++kb, ++it) {
           const int s = it % NSTAGE;
-          if (!ptx::mbar_wait_cluster(full_bar(s), (it / NSTAGE) & 1, abort_flag, global_abort)) {
+          if (!ptx::mbar_wait_cluster<HINT>(full_bar(s), (it / NSTAGE) & 1, abort_flag, global_abort)) {
             timeout(4); ok = false; break;
           }
           ptx::tc_fence_after();
