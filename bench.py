@@ -463,6 +463,9 @@ def main():
                      "flops_per_launch": flops_g1, "avg_launch_ms": g1_avg_s * 1e3, "launches": g1_launches,
                      "traffic": GEMM1_DRAM_TRAFFIC.get(cfg.name)},
         "ffn_tflops_layer": 6.0 * cfg.P * cfg.d * cfg.f * args.steps / (elapsed_ms * 1e-3) / 1e12,
+        "paper_context": "the paper reports only relative figures: up to 1.79x end-to-end training speedup over COMET "
+                         "(geomean 1.59x) on a SIMULATED 32-GPU GH200 NVL32 (BookSim2 + Accel-Sim, H200-configured "
+                         "GPUs, NVLink 4, FP8 GEMMs); no tokens/s, GB/s or TFLOP/s for this path, hence vs_baseline null",
     }
     if world == 1 and not args.lean:
         line["stages"] = stage_breakdown(cfg, t)

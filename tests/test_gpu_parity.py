@@ -28,6 +28,9 @@ SMALL = [
     # a single token; many tokens in a single expert pair tile boundary (257 rows: 128 + 128 + 1)
     synth.MoEConfig("T1", T=1, d=64, f=64, E=8, k=2, G=2, seed=9),
     synth.MoEConfig("rows257", T=257, d=64, f=192, E=2, k=2, G=1, seed=10),
+    # the paper's evaluation sweeps top-k over 8 / 16 / 32 (Table I): many slots per token, most in one group
+    synth.MoEConfig("topk16", T=130, d=128, f=64, E=64, k=16, G=8, score_fn=1, seed=13),
+    synth.MoEConfig("topk32", T=90, d=64, f=64, E=64, k=32, G=4, bias="locality", boost=2.0, seed=14),
     # long K: GEMM-1 takes its split-ring pipeline (K >= 6144), with a K tail (6216 = 97 * 64 + 8)
     synth.MoEConfig("longK", T=300, d=6216, f=72, E=3, k=2, G=3, seed=11),
 ]
