@@ -246,10 +246,17 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
         for n in ("route", "dispatch", "expert_ffn", "combine"):
             calls[n]()
 
-    seq_ms, fus_ms = [], []
+    # third variant: Combine inside GEMM-2's epilogue (fp32 reductions, o never written)
+    shape_epi = B.make_shape(cfg, B.MOE_FLAG_COMBINE_IN_EPILOGUE)
+
+    def layer_epilogue_combine():
+        B.moe_layer(shape_epi, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws)
+
+    seq_ms, fus_ms, epi_ms = [], [], []
     for _ in range(reps):
         seq_ms.append(timed(unfused_seq))
         fus_ms.append(timed(calls["layer_fused"]))
+        epi_ms.append(timed(layer_epilogue_combine))
     # in-layer (back to back, no idle gap) kernel times of the fused call
     for kn in kernels["layer_fused"]:
         B.moe_profile_enable(B.KERNEL_IDS[kn])
@@ -260,7 +267,9 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
         out["layer_fused"][kn + "_in_layer_ms"] = ms / max(n, 1)
     out["combine"]["in_layer_gbs"] = comb_bytes / out["layer_fused"]["combine_in_layer_ms"] / 1e6
     out["summary"] = {"unfused_sum_ms": unfused, "unfused_back_to_back_ms": float(np.median(seq_ms)),
-                      "fused_back_to_back_ms": float(np.median(fus_ms)), "fused_ms": out["layer_fused"]["ms"],
+                      "fused_back_to_back_ms": float(np.median(fus_ms)),
+                      "fused_epilogue_combine_back_to_back_ms": float(np.median(epi_ms)),
+                      "fused_ms": out["layer_fused"]["ms"],
                       "fused_tokens_per_s": T / out["layer_fused"]["ms"] * 1e3,
                       "n_disp": n_disp, "pairs": P, "dedup": 1.0 - n_disp / P,
                       "rows_per_expert_min": int(counts.min()), "rows_per_expert_max": int(counts.max()),

@@ -57,8 +57,19 @@ enum { MOE_WARN_NONFINITE_LOGIT = 1 };
 
 enum { MOE_SCORE_SOFTMAX = 0,      /* weights = softmax over the k selected keys          */
        MOE_SCORE_SIGMOID = 1 };    /* weights = sigmoid(key) renormalised over the k      */
-enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1 }; /* default (0): gate weight applied in GEMM-2's
+enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1,   /* default (0): gate weight applied in GEMM-2's
                                             epilogue, Combine un-weighted (Sec. III-C)    */
+       MOE_FLAG_COMBINE_IN_EPILOGUE = 2 }; /* moe_layer only: Combine runs inside GEMM-2's
+                                            epilogue (Sec. V, fused pipeline): every weighted
+                                            expert row is added into an fp32 accumulator row of
+                                            its token with vector reductions, o is never
+                                            written, a last pass rounds the accumulators to
+                                            bf16.  The k additions of a token then happen in
+                                            arrival order, so y may differ from the default
+                                            form in the last fp32 bit before rounding (not
+                                            run-to-run reproducible).  Excludes
+                                            MOE_FLAG_WEIGHT_IN_COMBINE; the stage entry points
+                                            moe_expert_ffn / moe_combine reject it.        */
 
 /* Shape of one layer.  Limits: 1 <= k <= min(E, 32); E <= 1024; E % G == 0;
  * d % 8 == 0; f % 8 == 0; T >= 0; T * max(k, G) < 2^31. */

@@ -44,7 +44,8 @@ WsPlan plan(const moe_shape_t& s) {
   p.mp_prefix = take((E + 1) * 4);
   p.wsplit = take(gate_split_bytes(s.d, s.E));
   p.h = take(P * (size_t)s.f * 2);
-  p.o = take(P * (size_t)s.d * 2);
+  // o [P, d] bf16, or the fp32 token accumulators [T, d] of the Combine-in-epilogue form
+  p.o = take((P * 2 > T * 4 ? P * 2 : T * 4) * (size_t)s.d);
   p.logits = take(T * E * 4);
   p.topk_idx = take(P * 4);
   p.topk_w = take(P * 4);
@@ -65,7 +66,8 @@ int check_shape(const moe_shape_t* s) {
   if (s == nullptr) return MOE_ERR_INVALID_ARG;
   if (s->T < 0 || s->d <= 0 || s->f <= 0 || s->E <= 0 || s->k <= 0 || s->G <= 0) return MOE_ERR_INVALID_ARG;
   if (s->score_fn != MOE_SCORE_SOFTMAX && s->score_fn != MOE_SCORE_SIGMOID) return MOE_ERR_INVALID_ARG;
-  if (s->flags & ~MOE_FLAG_WEIGHT_IN_COMBINE) return MOE_ERR_INVALID_ARG;
+  if (s->flags & ~(MOE_FLAG_WEIGHT_IN_COMBINE | MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
+  if ((s->flags & MOE_FLAG_WEIGHT_IN_COMBINE) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
   if (s->k > s->E || s->G > s->E || s->E % s->G != 0) return MOE_ERR_INVALID_ARG;
   if (s->k > 32 || s->E > 1024 || s->d % 8 != 0 || s->f % 8 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
   const long long kg = s->k > s->G ? s->k : s->G;
@@ -278,6 +280,7 @@ int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t*
   int rc = check_shape(shape);
   if (rc != MOE_OK) return rc;
   if (xg == nullptr || w1 == nullptr || w3 == nullptr || w2 == nullptr || o == nullptr) return MOE_ERR_INVALID_ARG;
+  if (shape->flags & MOE_FLAG_COMBINE_IN_EPILOGUE) return MOE_ERR_INVALID_ARG;   // a moe_layer option: o is the result here
   const bool in_combine = (shape->flags & MOE_FLAG_WEIGHT_IN_COMBINE) != 0;
   if (!in_combine && topk_w == nullptr) return MOE_ERR_INVALID_ARG;
   if ((rc = check_layout(layout)) != MOE_OK) return rc;
@@ -314,6 +317,7 @@ int moe_combine(const moe_shape_t* shape, const void* o, const moe_layout_t* lay
   int rc = check_shape(shape);
   if (rc != MOE_OK) return rc;
   if (o == nullptr || y == nullptr || topk_idx == nullptr) return MOE_ERR_INVALID_ARG;
+  if (shape->flags & MOE_FLAG_COMBINE_IN_EPILOGUE) return MOE_ERR_INVALID_ARG;
   if ((shape->flags & MOE_FLAG_WEIGHT_IN_COMBINE) && topk_w == nullptr) return MOE_ERR_INVALID_ARG;
   if ((rc = check_layout(layout)) != MOE_OK) return rc;
   if (!aligned(o, 128) || !aligned(y, 128) || !aligned(pg, 128) || !aligned(topk_idx, 16) || !aligned(topk_w, 16))
@@ -376,6 +380,14 @@ int moe_layer(const moe_shape_t* shape, const void* x, const float* w_gate, cons
   a.mt_prefix = at<int32_t>(ws, p.mt_prefix);
   a.mp_prefix = at<int32_t>(ws, p.mp_prefix);
   a.status = status;
+  if (s.flags & MOE_FLAG_COMBINE_IN_EPILOGUE) {
+    // o never materialises: GEMM-2 adds each weighted row into its token's fp32 accumulator
+    a.y_acc = at<float>(ws, p.o);
+    if (s.T > 0) TCMOE_CUDA(cudaMemsetAsync(a.y_acc, 0, (size_t)s.T * s.d * 4, st));
+    TCMOE_CUDA(launch_expert_ffn(s, a, st));
+    TCMOE_CUDA(launch_round_rows(s, a.y_acc, y, st));
+    return MOE_OK;
+  }
   TCMOE_CUDA(launch_expert_ffn(s, a, st));
   TCMOE_CUDA(launch_combine(s, a.o, L, idx, tw, nullptr, y, st));
   return MOE_OK;

@@ -55,6 +55,7 @@ cudaError_t launch_layout(const Shape& s, const int32_t* topk_idx, const Layout&
 cudaError_t launch_tile_prefix(const Shape& s, const int32_t* expert_counts, int32_t* mt_prefix, int32_t* mp_prefix,
                                cudaStream_t st);
 cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void* xg, cudaStream_t st);
+cudaError_t launch_round_rows(const Shape& s, const float* acc, void* y, cudaStream_t st);
 cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
                            const float* topk_w, void* pg, void* y, cudaStream_t st);
 // ffn.cu
@@ -64,7 +65,8 @@ struct FfnArgs {
   int gather_div;
   const void *w1, *w3, *w2;
   void* h;                    // [P, f] bf16 scratch
-  void* o;                    // [P, d] bf16 out
+  void* o;                    // [P, d] bf16 out (unused when y_acc is set)
+  float* y_acc;               // Combine in GEMM-2's epilogue: zeroed fp32 [T, d] accumulator, else NULL
   const float* topk_w;        // NULL: un-weighted epilogue
   const int32_t* row_pair;
   const int32_t* expert_offsets;

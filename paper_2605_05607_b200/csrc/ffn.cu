@@ -104,6 +104,8 @@ cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st)
   g2.N = s.d;
   g2.n_tiles = (s.d + 255) / 256;
   g2.status = a.status;
+  g2.y_acc = a.y_acc;
+  g2.y_div = s.k;
   return ffn::launch_gemm2(g2, m_w2, m_h, st);
 }
 

@@ -29,6 +29,8 @@ struct GemmParams {
                                 // 256-row CTA-pair tiles for GEMM-2)
   int E, K, N, n_tiles;
   int32_t* status;
+  float* y_acc;                 // GEMM-2 with Combine in its epilogue: fp32 [T, N] accumulator, token
+  int y_div;                    // of row r = row_pair[r] / y_div (NULL: rows go to `out`)
 };
 
 struct Tile {

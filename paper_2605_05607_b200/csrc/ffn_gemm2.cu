@@ -35,6 +35,10 @@ constexpr int BN_OUT = 256;
 constexpr uint32_t IDESC = idesc_bf16(2 * BM);
 constexpr uint32_t HINT = 4000;   // try_wait suspend-time hint (ns), see ptx::mbar_try_wait
 
+// RED = false: rows go to o (bf16), Combine is a later pass.  RED = true: Combine happens here
+// (Sec. V: the fused pipeline reduces expert outputs as GEMM-2 produces them): each weighted row is
+// added into the fp32 accumulator row of its token with vector reductions; o is never written.
+template <bool RED>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_h,
                  const GemmParams p) {
@@ -110,9 +114,15 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
       const bool valid = lrow < t.rows;
       const size_t grow = (size_t)(valid ? t.row0 + lrow : 0);
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UMMA_N);
-      __nv_bfloat16* orow = p.out + grow * (size_t)p.out_ld + t.n0;
+      __nv_bfloat16* orow = nullptr;
+      float* yrow = nullptr;
       float wr = 1.f;
-      if (valid && p.topk_w != nullptr) wr = __ldg(p.topk_w + __ldg(p.row_pair + grow));
+      if (valid) {
+        const int pair = __ldg(p.row_pair + grow);
+        if (p.topk_w != nullptr) wr = __ldg(p.topk_w + pair);
+        if (RED) yrow = p.y_acc + (size_t)(pair / p.y_div) * (size_t)p.N + t.n0;
+      }
+      if (!RED) orow = p.out + grow * (size_t)p.out_ld + t.n0;
 #pragma unroll 1
       for (int c = 0; c < 8; ++c) {
         uint32_t acc[32];
@@ -121,7 +131,15 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
         if (valid) {
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
-            if (t.n0 + c * 32 + v * 8 < p.N) {
+            if (RED) {
+              if (t.n0 + c * 32 + v * 8 < p.N) {
+                float* dst = yrow + c * 32 + v * 8;
+                ptx::red_add_v4(dst, wr * __uint_as_float(acc[v * 8]), wr * __uint_as_float(acc[v * 8 + 1]),
+                                wr * __uint_as_float(acc[v * 8 + 2]), wr * __uint_as_float(acc[v * 8 + 3]));
+                ptx::red_add_v4(dst + 4, wr * __uint_as_float(acc[v * 8 + 4]), wr * __uint_as_float(acc[v * 8 + 5]),
+                                wr * __uint_as_float(acc[v * 8 + 6]), wr * __uint_as_float(acc[v * 8 + 7]));
+              }
+            } else if (t.n0 + c * 32 + v * 8 < p.N) {
               uint4 q;
               uint32_t* qq = reinterpret_cast<uint32_t*>(&q);
 #pragma unroll
@@ -229,7 +247,7 @@ int pair_grid() {
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    if (cudaOccupancyMaxActiveClusters(&clusters, ffn_gemm2_kernel, &cfg) != cudaSuccess || clusters <= 0) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, ffn_gemm2_kernel<false>, &cfg) != cudaSuccess || clusters <= 0) {
       (void)cudaGetLastError();
       clusters = sm_count() / 2;
     }
@@ -244,12 +262,17 @@ cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUt
   static bool attr_set[MAX_DEVICES] = {};   // the attribute is per device
   const int dev = current_device();
   if (!attr_set[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(ffn_gemm2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
   }
   ProfileScope prof(KID_GEMM2, st);
-  ffn_gemm2_kernel<<<pair_grid(), THREADS, SMEM_BYTES, st>>>(m_w2, m_h, p);
+  if (p.y_acc != nullptr)
+    ffn_gemm2_kernel<true><<<pair_grid(), THREADS, SMEM_BYTES, st>>>(m_w2, m_h, p);
+  else
+    ffn_gemm2_kernel<false><<<pair_grid(), THREADS, SMEM_BYTES, st>>>(m_w2, m_h, p);
   return cudaGetLastError();
 }
 

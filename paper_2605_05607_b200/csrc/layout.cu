@@ -320,4 +320,33 @@ cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const
   return cudaGetLastError();
 }
 
+// Last step of the layer when Combine ran inside GEMM-2's epilogue: the fp32 token accumulators
+// become the bf16 output, 8 elements per thread.
+__global__ void __launch_bounds__(256) round_rows_kernel(const float4* __restrict__ acc, uint4* __restrict__ y,
+                                                         size_t n_vec) {
+  const size_t stride = (size_t)gridDim.x * blockDim.x;
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
+    const float4 a = __ldcs(acc + 2 * i), b = __ldcs(acc + 2 * i + 1);
+    uint4 q;
+    __nv_bfloat162 v;
+    v = __floats2bfloat162_rn(a.x, a.y); q.x = *reinterpret_cast<uint32_t*>(&v);
+    v = __floats2bfloat162_rn(a.z, a.w); q.y = *reinterpret_cast<uint32_t*>(&v);
+    v = __floats2bfloat162_rn(b.x, b.y); q.z = *reinterpret_cast<uint32_t*>(&v);
+    v = __floats2bfloat162_rn(b.z, b.w); q.w = *reinterpret_cast<uint32_t*>(&v);
+    y[i] = q;
+  }
+}
+
+cudaError_t launch_round_rows(const Shape& s, const float* acc, void* y, cudaStream_t st) {
+  const size_t n_vec = (size_t)s.T * s.d / 8;
+  if (n_vec == 0) return cudaSuccess;
+  size_t blocks = (n_vec + 255) / 256;
+  const size_t cap = (size_t)sm_count() * 16;
+  if (blocks > cap) blocks = cap;
+  ProfileScope prof(KID_COMBINE, st);
+  round_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(acc), static_cast<uint4*>(y),
+                                                      n_vec);
+  return cudaGetLastError();
+}
+
 }  // namespace tcmoe

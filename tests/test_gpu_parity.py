@@ -99,6 +99,19 @@ def test_fused_layer_matches_oracle_and_staged(cfg):
     run.layer(y=y3)
     assert torch.equal(y3, y2)
     assert run.status()[0] == 0
+    # Combine inside GEMM-2's epilogue (fp32 reductions in arrival order).  The default form rounds
+    # every o row to bf16 before summing, this one sums unrounded fp32 rows: the two agree within
+    # that rounding (k terms, 2^-9 relative each), and both meet the output bar against the oracle
+    if "wcombine" not in cfg.name:
+        run_e = H.Run(cfg, B.MOE_FLAG_COMBINE_IN_EPILOGUE, inputs=run.t)
+        for _ in range(2):   # twice: the accumulators are cleared by every call
+            y4 = torch.full_like(run.y, 7.0)
+            run_e.layer(y=y4)
+        y_epi = O.bf16_to_f64(H.bf16_host(y4)[: cfg.T])
+        H.assert_close_out(y_epi, y_def, "epilogue-combine y")
+        mx, mean = H.out_errors(y_epi, y_fused)
+        assert mx <= 1e-2 and mean <= 3e-3, f"epilogue-combine y vs default fused y: {mx:.2e} {mean:.2e}"
+        assert run_e.status()[0] == 0
 
 
 def test_topk_ties_lowest_index_wins():
@@ -172,6 +185,15 @@ def test_degenerate_and_error_paths():
     torch.cuda.synchronize()
     assert run.status()[0] == 0
     assert run.lay.expert_offsets[:5].tolist() == [0] * 5
+    # flag combinations without meaning are refused before anything is launched
+    both = B.MOE_FLAG_WEIGHT_IN_COMBINE | B.MOE_FLAG_COMBINE_IN_EPILOGUE
+    with pytest.raises(B.MoEError):
+        B.alloc_workspace(B.make_shape(cfg.with_(T=8), both))
+    run_e = H.Run(cfg.with_(T=8), B.MOE_FLAG_COMBINE_IN_EPILOGUE, inputs=run.t)
+    with pytest.raises(B.MoEError):
+        run_e.ffn()
+    with pytest.raises(B.MoEError):
+        run_e.combine()
     # an out-of-range expert index is reported, not dereferenced
     cfg = synth.MoEConfig("badidx", T=40, d=64, f=64, E=4, k=2, G=2)
     run = H.Run(cfg, inputs=synth.make_routing_inputs(cfg, "cuda") | {"w1": None, "w3": None, "w2": None})
