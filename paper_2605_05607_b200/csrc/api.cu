@@ -362,9 +362,12 @@ int moe_layer(const moe_shape_t* shape, const void* x, const float* w_gate, cons
   }
   // gate
   TCMOE_CUDA(launch_gate_logits(s, x, w_gate, lg, at<void>(ws, p.wsplit), status, st));
-  TCMOE_CUDA(launch_topk(s, lg, logit_bias, bias_row_stride, idx, tw, status, st));
+  // the top-k kernel also zeroes the bitmasks of the layout builder (emask and gmask are adjacent)
+  const LayoutScratch sc = scratch(ws, p);
+  TCMOE_CUDA(launch_topk(s, lg, logit_bias, bias_row_stride, idx, tw, status, st, sc.emask,
+                         (size_t)(s.E + s.G) * sc.W));
   // layout only: the dispatched copy xg is never written, GEMM-1 gathers token rows from x
-  TCMOE_CUDA(launch_layout(s, idx, L, scratch(ws, p), status, st));
+  TCMOE_CUDA(launch_layout(s, idx, L, sc, status, st, /*masks_cleared=*/s.T > 0));
   FfnArgs a{};
   a.a_src = x;
   a.gather_idx = L.row_pair;   // token of expert row r = row_pair[r] / k

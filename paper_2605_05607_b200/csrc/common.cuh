@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <utility>
 
 namespace tcmoe {
 
@@ -19,6 +20,33 @@ __device__ __forceinline__ void report_error(int32_t* status, int code, int wher
     status[ST_DETAIL] = detail;
     status[ST_AUX] = aux;
   }
+}
+
+// ---- programmatic dependent launch ------------------------------------------------------------
+// Every kernel of the library is launched with programmatic stream serialisation and starts with
+// grid_dependency_sync(): set-up that touches no global data (barrier init, TMEM allocation,
+// tensor-map prefetch) may run while the previous kernel of the stream drains; nothing is read
+// from or written to global memory before the previous kernel has completed and flushed, so
+// results are those of plain stream order.  The call also lets the next kernel of the stream
+// begin its own set-up.
+__device__ __forceinline__ void grid_dependency_sync() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
 }
 
 // ---- problem description passed to the launchers ---------------------------------------------
@@ -48,10 +76,11 @@ cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gat
                                int32_t* status, cudaStream_t st);
 // route.cu
 cudaError_t launch_topk(const Shape& s, const float* logits, const float* bias, int64_t bias_stride,
-                        int32_t* topk_idx, float* topk_w, int32_t* status, cudaStream_t st);
+                        int32_t* topk_idx, float* topk_w, int32_t* status, cudaStream_t st,
+                        uint32_t* clear = nullptr, size_t clear_words = 0);   // clear: words zeroed on the side
 // layout.cu
 cudaError_t launch_layout(const Shape& s, const int32_t* topk_idx, const Layout& L, const LayoutScratch& sc,
-                          int32_t* status, cudaStream_t st);
+                          int32_t* status, cudaStream_t st, bool masks_cleared = false);
 cudaError_t launch_tile_prefix(const Shape& s, const int32_t* expert_counts, int32_t* mt_prefix, int32_t* mp_prefix,
                                cudaStream_t st);
 cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void* xg, cudaStream_t st);

@@ -67,12 +67,7 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  for (int i = threadIdx.x; i <= p.E; i += blockDim.x) {
-    tp_s[i] = p.tile_prefix[i];
-    eoff_s[i] = p.expert_offsets[i];
-  }
   if (threadIdx.x == 0) {
-    *abort_s = p.status[ST_ABORT];
     for (int s = 0; s < NA; ++s) {
       ptx::mbar_init(afull_bar(s), SPLIT ? 4 : 5);   // one lane per gather warp (+ the TMA thread when joint)
       ptx::mbar_init(aempty_bar(s), 1);              // tcgen05.commit
@@ -97,6 +92,12 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
     ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
     ptx::tmem_relinquish();
   }
+  grid_dependency_sync();   // nothing above touches global data
+  for (int i = threadIdx.x; i <= p.E; i += blockDim.x) {
+    tp_s[i] = p.tile_prefix[i];
+    eoff_s[i] = p.expert_offsets[i];
+  }
+  if (threadIdx.x == 0) *abort_s = p.status[ST_ABORT];
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -290,9 +291,8 @@ cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUt
     attr_set[dev] = true;
   }
   ProfileScope prof(KID_GEMM1, st);
-  if (p.K >= 6144) ffn_gemm1_kernel<true><<<sm_count(), THREADS, SMEM_BYTES, st>>>(m_w1, m_w3, p);
-  else ffn_gemm1_kernel<false><<<sm_count(), THREADS, SMEM_BYTES, st>>>(m_w1, m_w3, p);
-  return cudaGetLastError();
+  if (p.K >= 6144) return launch_pdl(ffn_gemm1_kernel<true>, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);
+  return launch_pdl(ffn_gemm1_kernel<false>, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);
 }
 
 }  // namespace ffn

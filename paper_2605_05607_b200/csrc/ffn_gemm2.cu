@@ -61,12 +61,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
   const int rank = (int)ptx::cluster_ctarank();
   const int cluster_id = blockIdx.x >> 1, num_clusters = gridDim.x >> 1;
 
-  for (int i = threadIdx.x; i <= p.E; i += blockDim.x) {
-    tp_s[i] = p.tile_prefix[i];
-    eoff_s[i] = p.expert_offsets[i];
-  }
   if (threadIdx.x == 0) {
-    *abort_s = p.status[ST_ABORT];
     for (int s = 0; s < NSTAGE; ++s) {
       ptx::mbar_init(full_bar(s), 1);       // leader TMA thread (expect_tx for both CTAs)
       ptx::mbar_init(empty_bar(s), 1);      // tcgen05.commit
@@ -85,6 +80,12 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
     ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), 512);
     ptx::tmem_relinquish_pair();
   }
+  grid_dependency_sync();   // nothing above touches global data
+  for (int i = threadIdx.x; i <= p.E; i += blockDim.x) {
+    tp_s[i] = p.tile_prefix[i];
+    eoff_s[i] = p.expert_offsets[i];
+  }
+  if (threadIdx.x == 0) *abort_s = p.status[ST_ABORT];
   ptx::tc_fence_before();
   __syncthreads();
   ptx::cluster_sync();   // the peer's barriers are initialised before anything signals them
@@ -269,11 +270,8 @@ cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUt
     attr_set[dev] = true;
   }
   ProfileScope prof(KID_GEMM2, st);
-  if (p.y_acc != nullptr)
-    ffn_gemm2_kernel<true><<<pair_grid(), THREADS, SMEM_BYTES, st>>>(m_w2, m_h, p);
-  else
-    ffn_gemm2_kernel<false><<<pair_grid(), THREADS, SMEM_BYTES, st>>>(m_w2, m_h, p);
-  return cudaGetLastError();
+  if (p.y_acc != nullptr) return launch_pdl(ffn_gemm2_kernel<true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
+  return launch_pdl(ffn_gemm2_kernel<false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
 }
 
 }  // namespace ffn

@@ -32,6 +32,7 @@ constexpr int THREADS = 192;
 // w_gate fp32 [d, E] -> bf16 [3, d, Epad]: hi, mid, lo terms, zero in the padding columns
 __global__ void __launch_bounds__(256) split_gate_kernel(const float* __restrict__ wg, __nv_bfloat16* __restrict__ out,
                                                          int d, int E, int Epad) {
+  grid_dependency_sync();
   const size_t n = (size_t)d * Epad;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     const int row = (int)(i / Epad), col = (int)(i % Epad);
@@ -80,7 +81,6 @@ gate_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   const int iters = sbs ? p.KB : 3 * p.KB;
 
   if (threadIdx.x == 0) {
-    *abort_s = p.status[ST_ABORT];
     for (int s = 0; s < MAX_STAGES; ++s) {
       ptx::mbar_init(full_bar(s), 1);
       ptx::mbar_init(empty_bar(s), 1);
@@ -96,6 +96,8 @@ gate_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
     ptx::tmem_alloc(ptx::smem_u32(tmem_slot), 512);
     ptx::tmem_relinquish();
   }
+  grid_dependency_sync();   // nothing above touches global data
+  if (threadIdx.x == 0) *abort_s = p.status[ST_ABORT];
   ptx::tc_fence_before();
   __syncthreads();
   ptx::tc_fence_after();
@@ -269,7 +271,9 @@ cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gat
   const size_t n = (size_t)s.d * Epad;
   int sb = (int)((n + 255) / 256);
   if (sb > sm_count() * 8) sb = sm_count() * 8;
-  split_gate_kernel<<<sb, 256, 0, st>>>(w_gate, static_cast<__nv_bfloat16*>(wsplit), s.d, s.E, Epad);
+  cudaError_t err = launch_pdl(split_gate_kernel, sb, 256, 0, st, w_gate, static_cast<__nv_bfloat16*>(wsplit), s.d, s.E,
+                               Epad);
+  if (err != cudaSuccess) return err;
   GateParams p;
   p.logits = logits;
   p.T = s.T;
@@ -279,8 +283,7 @@ cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gat
   p.side_by_side = s.E <= 128 ? 1 : 0;
   p.status = status;
   const int grid = ((s.T + BM - 1) / BM) * p.n_tiles;
-  gate_umma_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(m_x, m_w, p);
-  return cudaGetLastError();
+  return launch_pdl(gate_umma_kernel, grid, THREADS, SMEM_BYTES, st, m_x, m_w, p);
 }
 
 }  // namespace tcmoe

@@ -17,6 +17,7 @@ namespace tcmoe {
 __global__ void __launch_bounds__(256) build_masks_kernel(const int32_t* __restrict__ topk_idx, uint32_t* emask,
                                                           uint32_t* gmask, int T, int E, int k, int m, int W,
                                                           int32_t* status) {
+  grid_dependency_sync();
   const int t = blockIdx.x * blockDim.x + threadIdx.x;  // warp w covers tokens 32w .. 32w+31
   const int lane = threadIdx.x & 31;
   const int word = t >> 5;
@@ -41,6 +42,7 @@ __global__ void __launch_bounds__(256) scan_masks_kernel(const uint32_t* __restr
                                                          const uint32_t* __restrict__ gmask, int32_t* eprefix,
                                                          int32_t* gprefix, int32_t* expert_counts,
                                                          int32_t* group_counts, int E, int W) {
+  grid_dependency_sync();
   __shared__ int warp_sum[8];
   __shared__ int running_s;
   const int row = blockIdx.x;
@@ -79,6 +81,7 @@ __global__ void __launch_bounds__(1024) offsets_kernel(const int32_t* __restrict
                                                        const int32_t* __restrict__ group_counts,
                                                        int32_t* expert_offsets, int32_t* group_offsets,
                                                        int32_t* mt_prefix, int32_t* mp_prefix, int E, int G) {
+  grid_dependency_sync();
   __shared__ int buf[4][1024];
   const int i = threadIdx.x;
   const int ce = (i < E) ? expert_counts[i] : 0;
@@ -103,6 +106,7 @@ __global__ void __launch_bounds__(1024) offsets_kernel(const int32_t* __restrict
 // ---- K2d: ranks -> row tables ----------------------------------------------------------------
 __global__ void __launch_bounds__(256) fill_layout_kernel(const int32_t* __restrict__ topk_idx, Layout L,
                                                           LayoutScratch sc, int T, int E, int k, int G, int m) {
+  grid_dependency_sync();
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= T) return;
   const int word = t >> 5;
@@ -133,6 +137,7 @@ __global__ void __launch_bounds__(256) fill_layout_kernel(const int32_t* __restr
 // exclusive prefixes of 128-row tiles and 256-row pair tiles per expert, from the counts alone
 __global__ void __launch_bounds__(1024) tile_prefix_kernel(const int32_t* __restrict__ expert_counts,
                                                            int32_t* mt_prefix, int32_t* mp_prefix, int E) {
+  grid_dependency_sync();
   __shared__ int buf[2][1024];
   const int i = threadIdx.x;
   const int c = (i < E) ? expert_counts[i] : 0;
@@ -152,24 +157,28 @@ __global__ void __launch_bounds__(1024) tile_prefix_kernel(const int32_t* __rest
 
 cudaError_t launch_tile_prefix(const Shape& s, const int32_t* expert_counts, int32_t* mt_prefix, int32_t* mp_prefix,
                                cudaStream_t st) {
-  tile_prefix_kernel<<<1, 1024, 0, st>>>(expert_counts, mt_prefix, mp_prefix, s.E);
-  return cudaGetLastError();
+  return launch_pdl(tile_prefix_kernel, 1, 1024, 0, st, expert_counts, mt_prefix, mp_prefix, s.E);
 }
 
 cudaError_t launch_layout(const Shape& s, const int32_t* topk_idx, const Layout& L, const LayoutScratch& sc,
-                          int32_t* status, cudaStream_t st) {
+                          int32_t* status, cudaStream_t st, bool masks_cleared) {
   const int m = s.E / s.G;
   cudaError_t err;
-  if ((err = cudaMemsetAsync(sc.emask, 0, sizeof(uint32_t) * (size_t)(s.E + s.G) * sc.W, st)) != cudaSuccess)
+  if (!masks_cleared &&
+      (err = cudaMemsetAsync(sc.emask, 0, sizeof(uint32_t) * (size_t)(s.E + s.G) * sc.W, st)) != cudaSuccess)
     return err;  // emask and gmask are adjacent
   const int tb = (s.T + 255) / 256;
-  if (s.T > 0) build_masks_kernel<<<tb, 256, 0, st>>>(topk_idx, sc.emask, sc.gmask, s.T, s.E, s.k, m, sc.W, status);
-  scan_masks_kernel<<<s.E + s.G, 256, 0, st>>>(sc.emask, sc.gmask, sc.eprefix, sc.gprefix, L.expert_counts,
-                                                L.group_counts, s.E, sc.W);
-  offsets_kernel<<<1, 1024, 0, st>>>(L.expert_counts, L.group_counts, L.expert_offsets, L.group_offsets,
-                                     sc.mt_prefix, sc.mp_prefix, s.E, s.G);
-  if (s.T > 0) fill_layout_kernel<<<tb, 256, 0, st>>>(topk_idx, L, sc, s.T, s.E, s.k, s.G, m);
-  return cudaGetLastError();
+  if (s.T > 0 && (err = launch_pdl(build_masks_kernel, tb, 256, 0, st, topk_idx, sc.emask, sc.gmask, s.T, s.E, s.k,
+                                   m, sc.W, status)) != cudaSuccess)
+    return err;
+  if ((err = launch_pdl(scan_masks_kernel, s.E + s.G, 256, 0, st, sc.emask, sc.gmask, sc.eprefix, sc.gprefix,
+                        L.expert_counts, L.group_counts, s.E, sc.W)) != cudaSuccess)
+    return err;
+  if ((err = launch_pdl(offsets_kernel, 1, 1024, 0, st, L.expert_counts, L.group_counts, L.expert_offsets,
+                        L.group_offsets, sc.mt_prefix, sc.mp_prefix, s.E, s.G)) != cudaSuccess)
+    return err;
+  if (s.T > 0) return launch_pdl(fill_layout_kernel, tb, 256, 0, st, topk_idx, L, sc, s.T, s.E, s.k, s.G, m);
+  return cudaSuccess;
 }
 
 // ---- K3: dispatch ------------------------------------------------------------------------------
@@ -179,6 +188,7 @@ __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__
                                                        const int32_t* __restrict__ al,
                                                        const int32_t* __restrict__ group_offsets, int T, int G,
                                                        int vec_per_row) {
+  grid_dependency_sync();
   const int lane = threadIdx.x & 31;
   const int wpb = blockDim.x >> 5;
   for (int t = blockIdx.x * wpb + (threadIdx.x >> 5); t < T; t += gridDim.x * wpb) {
@@ -219,9 +229,8 @@ cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void
   const int cap = sm_count() * 8;
   if (blocks > cap) blocks = cap;
   ProfileScope prof(KID_DISPATCH, st);
-  dispatch_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(x), static_cast<uint4*>(xg), L.al,
-                                          L.group_offsets, s.T, s.G, s.d / 8);
-  return cudaGetLastError();
+  return launch_pdl(dispatch_kernel, blocks, 256, 0, st, static_cast<const uint4*>(x), static_cast<uint4*>(xg), L.al,
+                    L.group_offsets, s.T, s.G, s.d / 8);
 }
 
 // ---- K5: combine -----------------------------------------------------------------------------
@@ -252,6 +261,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
                                                       const int32_t* __restrict__ al,
                                                       const int32_t* __restrict__ group_offsets, int T, int k, int m,
                                                       int vec_per_row, int weighted) {
+  grid_dependency_sync();
   __shared__ int s_row[8][32];   // per warp: expert-sorted row of the slot at sorted position p
   __shared__ int s_dst[8][32];   // dispatched row (t, g) of that slot's group
   __shared__ float s_w[8][32];
@@ -314,16 +324,16 @@ cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const
   const int cap = sm_count() * 8;
   if (blocks > cap) blocks = cap;
   ProfileScope prof(KID_COMBINE, st);
-  combine_kernel<<<blocks, 256, 0, st>>>(static_cast<const uint4*>(o), static_cast<uint4*>(y),
-                                         static_cast<uint4*>(pg), topk_idx, topk_w, L.pair_row, L.al, L.group_offsets,
-                                         s.T, s.k, s.E / s.G, s.d / 8, (s.flags & 1) ? 1 : 0);
-  return cudaGetLastError();
+  return launch_pdl(combine_kernel, blocks, 256, 0, st, static_cast<const uint4*>(o), static_cast<uint4*>(y),
+                    static_cast<uint4*>(pg), topk_idx, topk_w, L.pair_row, L.al, L.group_offsets, s.T, s.k, s.E / s.G,
+                    s.d / 8, (s.flags & 1) ? 1 : 0);
 }
 
 // Last step of the layer when Combine ran inside GEMM-2's epilogue: the fp32 token accumulators
 // become the bf16 output, 8 elements per thread.
 __global__ void __launch_bounds__(256) round_rows_kernel(const float4* __restrict__ acc, uint4* __restrict__ y,
                                                          size_t n_vec) {
+  grid_dependency_sync();
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += stride) {
     const float4 a = __ldcs(acc + 2 * i), b = __ldcs(acc + 2 * i + 1);
@@ -344,9 +354,8 @@ cudaError_t launch_round_rows(const Shape& s, const float* acc, void* y, cudaStr
   const size_t cap = (size_t)sm_count() * 16;
   if (blocks > cap) blocks = cap;
   ProfileScope prof(KID_COMBINE, st);
-  round_rows_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(acc), static_cast<uint4*>(y),
-                                                      n_vec);
-  return cudaGetLastError();
+  return launch_pdl(round_rows_kernel, (unsigned)blocks, 256, 0, st, reinterpret_cast<const float4*>(acc),
+                    static_cast<uint4*>(y), n_vec);
 }
 
 }  // namespace tcmoe

@@ -31,7 +31,12 @@ template <int KPL>
 __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ logits, const float* __restrict__ bias,
                                                    long long bias_stride, int32_t* __restrict__ topk_idx,
                                                    float* __restrict__ topk_w, int T, int E, int k, int score_fn,
-                                                   int32_t* status) {
+                                                   int32_t* status, uint32_t* clear, size_t clear_words) {
+  grid_dependency_sync();
+  // optional side job for the fused layer: zero the membership bitmasks of the layout builder that
+  // runs next, so that no memset sits between this kernel and it
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < clear_words; i += (size_t)gridDim.x * blockDim.x)
+    clear[i] = 0u;
   const int lane = threadIdx.x & 31;
   const int warps_per_block = blockDim.x >> 5;
   bool nonfinite = false;
@@ -82,7 +87,8 @@ __global__ void __launch_bounds__(256) topk_kernel(const float* __restrict__ log
 }
 
 cudaError_t launch_topk(const Shape& s, const float* logits, const float* bias, int64_t bias_stride,
-                        int32_t* topk_idx, float* topk_w, int32_t* status, cudaStream_t st) {
+                        int32_t* topk_idx, float* topk_w, int32_t* status, cudaStream_t st, uint32_t* clear,
+                        size_t clear_words) {
   if (s.T == 0) return cudaSuccess;
   const int warps = 8;
   int blocks = (s.T + warps - 1) / warps;
@@ -90,17 +96,16 @@ cudaError_t launch_topk(const Shape& s, const float* logits, const float* bias, 
   if (blocks > cap) blocks = cap;
   const int kpl = (s.E + 31) / 32;
   ProfileScope prof(KID_TOPK, st);
-#define TCMOE_TOPK(KPL)                                                                                        \
-  topk_kernel<KPL><<<blocks, warps * 32, 0, st>>>(logits, bias, (long long)bias_stride, topk_idx, topk_w, s.T, \
-                                                  s.E, s.k, s.score_fn, status)
-  if (kpl <= 1) TCMOE_TOPK(1);
-  else if (kpl <= 2) TCMOE_TOPK(2);
-  else if (kpl <= 4) TCMOE_TOPK(4);
-  else if (kpl <= 8) TCMOE_TOPK(8);
-  else if (kpl <= 16) TCMOE_TOPK(16);
-  else TCMOE_TOPK(32);
+#define TCMOE_TOPK(KPL)                                                                                      \
+  launch_pdl(topk_kernel<KPL>, blocks, warps * 32, 0, st, logits, bias, (long long)bias_stride, topk_idx, topk_w, \
+             s.T, s.E, s.k, s.score_fn, status, clear, clear_words)
+  if (kpl <= 1) return TCMOE_TOPK(1);
+  if (kpl <= 2) return TCMOE_TOPK(2);
+  if (kpl <= 4) return TCMOE_TOPK(4);
+  if (kpl <= 8) return TCMOE_TOPK(8);
+  if (kpl <= 16) return TCMOE_TOPK(16);
+  return TCMOE_TOPK(32);
 #undef TCMOE_TOPK
-  return cudaGetLastError();
 }
 
 }  // namespace tcmoe
