@@ -266,6 +266,8 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
         B.moe_profile_enable(0)
         out["layer_fused"][kn + "_in_layer_ms"] = ms / max(n, 1)
     out["combine"]["in_layer_gbs"] = comb_bytes / out["layer_fused"]["combine_in_layer_ms"] / 1e6
+    out["inputs"] = {"seed": cfg.seed, "sub_streams": "seed*1000 + tensor id",
+                     "checksums": {n: synth.tensor_checksum(t[n]) for n in ("x", "w_gate", "bias", "w1", "w3", "w2")}}
     out["summary"] = {"unfused_sum_ms": unfused, "unfused_back_to_back_ms": float(np.median(seq_ms)),
                       "fused_back_to_back_ms": float(np.median(fus_ms)),
                       "fused_epilogue_combine_back_to_back_ms": float(np.median(epi_ms)),

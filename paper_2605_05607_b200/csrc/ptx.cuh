@@ -86,7 +86,7 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
   return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
 }
 
-// ---- TMA tiled loads (no multicast) -------------------------------------------------------------
+// ---- TMA tiled loads, one destination CTA each -------------------------------------------------------------
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* map, uint32_t bar, int c0, int c1) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"

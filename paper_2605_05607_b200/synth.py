@@ -139,6 +139,20 @@ def bits_to_bf16(a: np.ndarray, device="cpu") -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(a).view(np.int16)).view(torch.bfloat16).to(device)
 
 
+def tensor_checksum(t: Optional[torch.Tensor]) -> Optional[int]:
+    """Sum of the tensor's raw 16-bit words mod 2^61 - 1 (position-independent, cheap on any
+    device, chunked so that a 22 GB weight tensor needs no large temporary): identifies the seeded
+    inputs of a run in reports."""
+    if t is None:
+        return None
+    words = t.contiguous().view(-1).view(torch.int16)
+    total = 0
+    step = 1 << 28
+    for i in range(0, words.numel(), step):
+        total += int((words[i:i + step].to(torch.int32) & 0xFFFF).sum(dtype=torch.int64).item())
+    return total % ((1 << 61) - 1)
+
+
 def sample_tokens(cfg: MoEConfig, n: int, seed: int = 12345) -> np.ndarray:
     """Deterministic token sample for full-size output checks: the first and last
     64 tokens plus a seeded choice of the rest, ascending, without repeats."""
