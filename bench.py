@@ -294,7 +294,11 @@ def main():
     ap.add_argument("--steps", type=int, default=None,
                     help="timed steps (default 200: ~0.5 s on C2, long enough for clock samples; reference arm: 8)")
     ap.add_argument("--warmup", type=int, default=None, help="untimed warm-up steps (default 10; reference arm: 2)")
-    ap.add_argument("--config", default="C2", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--config", default="C2", choices=sorted(synth.ALL_CONFIGS),
+                    help="C1..C5b: the benchmark configurations; S8..L32: the paper's Small/Medium/Large shapes "
+                         "at top-k 8/16/32 (Table 'Model Configurations')")
+    ap.add_argument("--paper-shapes", action="store_true",
+                    help="with --report: also run the nine Small/Medium/Large x top-k shapes")
     ap.add_argument("--shape", default=None, metavar="T,d,f,E,k,G",
                     help="override the sizes of --config (keeps its score function and router bias); "
                          "for profiler captures of a slice that fits the capture size rules")
@@ -316,7 +320,7 @@ def main():
     if args.warmup is None:
         args.warmup = 10 if args.impl == "tcmoe" else 2
     args.warmup = max(args.warmup, 3) if args.impl == "tcmoe" else args.warmup
-    cfg = synth.CONFIGS[args.config]
+    cfg = synth.ALL_CONFIGS[args.config]
     if args.shape:
         T, d, f, E, k, G = (int(v) for v in args.shape.split(","))
         cfg = cfg.with_(name=f"{cfg.name}-slice", T=T, d=d, f=f, E=E, k=k, G=G)
@@ -484,7 +488,7 @@ def main():
         report = {cfg.name: line["stages"]}
         del t
         torch.cuda.empty_cache()
-        for name, c in synth.CONFIGS.items():
+        for name, c in (synth.ALL_CONFIGS if args.paper_shapes else synth.CONFIGS).items():
             if name != cfg.name:
                 tt = synth.make_inputs(c, "cuda")
                 report[name] = stage_breakdown(c, tt)

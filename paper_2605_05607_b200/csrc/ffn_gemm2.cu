@@ -29,7 +29,9 @@ constexpr int A_BYTES = BM * BK * 2;            // 16 KiB: this CTA's 128 rows
 constexpr int B_BYTES = (UMMA_N / 2) * BK * 2;  // 16 KiB: this CTA's half of the B tile (two 64-column slabs)
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int NUM_BARS = 2 * NSTAGE + 4;
-constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + 2 * (MAX_E + 1) * 4;
+constexpr int STAGE_OUT_WARP = 32 * 144;          // epilogue transpose buffer of one warp: 32 rows x (128 + 16) bytes
+constexpr int TABLE_BYTES = (2 * (MAX_E + 1) * 4 + 15) & ~15;
+constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + TABLE_BYTES + 4 * STAGE_OUT_WARP;
 constexpr int THREADS = 192;
 constexpr int BN_OUT = 256;
 constexpr uint32_t IDESC = idesc_bf16(2 * BM);
@@ -49,6 +51,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
   int* abort_s = reinterpret_cast<int*>(tmem_slot + 1);
   int* tp_s = reinterpret_cast<int*>(tmem_slot + 16);
   int* eoff_s = tp_s + (MAX_E + 1);
+  const uint32_t stage_base = ptx::smem_u32(tp_s) + TABLE_BYTES;   // 16-byte aligned
 
   const uint32_t smem_base = ptx::smem_u32(smem);
   const uint32_t bar_base = ptx::smem_u32(bars);
@@ -115,7 +118,6 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
       const bool valid = lrow < t.rows;
       const size_t grow = (size_t)(valid ? t.row0 + lrow : 0);
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UMMA_N);
-      __nv_bfloat16* orow = nullptr;
       float* yrow = nullptr;
       float wr = 1.f;
       if (valid) {
@@ -123,16 +125,15 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
         if (p.topk_w != nullptr) wr = __ldg(p.topk_w + pair);
         if (RED) yrow = p.y_acc + (size_t)(pair / p.y_div) * (size_t)p.N + t.n0;
       }
-      if (!RED) orow = p.out + grow * (size_t)p.out_ld + t.n0;
+      if (RED) {
 #pragma unroll 1
-      for (int c = 0; c < 8; ++c) {
-        uint32_t acc[32];
-        ptx::tmem_ld32(taddr + c * 32, acc);
-        ptx::tmem_ld_wait();
-        if (valid) {
+        for (int c = 0; c < 8; ++c) {
+          uint32_t acc[32];
+          ptx::tmem_ld32(taddr + c * 32, acc);
+          ptx::tmem_ld_wait();
+          if (valid) {
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            if (RED) {
+            for (int v = 0; v < 4; ++v) {
               if (t.n0 + c * 32 + v * 8 < p.N) {
                 float* dst = yrow + c * 32 + v * 8;
                 ptx::red_add_v4(dst, wr * __uint_as_float(acc[v * 8]), wr * __uint_as_float(acc[v * 8 + 1]),
@@ -140,17 +141,49 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
                 ptx::red_add_v4(dst + 4, wr * __uint_as_float(acc[v * 8 + 4]), wr * __uint_as_float(acc[v * 8 + 5]),
                                 wr * __uint_as_float(acc[v * 8 + 6]), wr * __uint_as_float(acc[v * 8 + 7]));
               }
-            } else if (t.n0 + c * 32 + v * 8 < p.N) {
-              uint4 q;
-              uint32_t* qq = reinterpret_cast<uint32_t*>(&q);
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const int j = v * 8 + 2 * i;
-                qq[i] = pack2(wr * __uint_as_float(acc[j]), wr * __uint_as_float(acc[j + 1]));
-              }
-              *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = q;
             }
           }
+        }
+      } else {
+        // A thread owns one accumulator row, but 32 threads storing 16 bytes each to 32 different
+        // rows cost 32 memory transactions per instruction.  The warp therefore transposes 64
+        // columns at a time through shared memory (rows padded to 144 bytes: conflict-free both
+        // ways) and stores whole 128-byte row segments, 8 lanes per row, 4 rows per instruction.
+        const uint32_t stage = stage_base + (uint32_t)(warp * STAGE_OUT_WARP);
+        const int srow = lane >> 3, piece = lane & 7;
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t acc0[32], acc1[32];
+          ptx::tmem_ld32(taddr + cc * 64, acc0);
+          ptx::tmem_ld32(taddr + cc * 64 + 32, acc1);
+          ptx::tmem_ld_wait_on(acc0);
+          ptx::tmem_ld_wait_on(acc1);
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            ptx::st_shared_v4(stage + lane * 144 + v * 16,
+                              pack2(wr * __uint_as_float(acc0[v * 8]), wr * __uint_as_float(acc0[v * 8 + 1])),
+                              pack2(wr * __uint_as_float(acc0[v * 8 + 2]), wr * __uint_as_float(acc0[v * 8 + 3])),
+                              pack2(wr * __uint_as_float(acc0[v * 8 + 4]), wr * __uint_as_float(acc0[v * 8 + 5])),
+                              pack2(wr * __uint_as_float(acc0[v * 8 + 6]), wr * __uint_as_float(acc0[v * 8 + 7])));
+            ptx::st_shared_v4(stage + lane * 144 + 64 + v * 16,
+                              pack2(wr * __uint_as_float(acc1[v * 8]), wr * __uint_as_float(acc1[v * 8 + 1])),
+                              pack2(wr * __uint_as_float(acc1[v * 8 + 2]), wr * __uint_as_float(acc1[v * 8 + 3])),
+                              pack2(wr * __uint_as_float(acc1[v * 8 + 4]), wr * __uint_as_float(acc1[v * 8 + 5])),
+                              pack2(wr * __uint_as_float(acc1[v * 8 + 6]), wr * __uint_as_float(acc1[v * 8 + 7])));
+          }
+          __syncwarp();
+          const int col = t.n0 + cc * 64 + piece * 8;
+          if (col < p.N) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int r = i * 4 + srow;           // row of this warp's 32
+              if (warp * 32 + r < t.rows) {
+                const uint4 q = ptx::ld_shared_v4(stage + r * 144 + piece * 16);
+                *reinterpret_cast<uint4*>(p.out + (size_t)(t.row0 + warp * 32 + r) * (size_t)p.out_ld + col) = q;
+              }
+            }
+          }
+          __syncwarp();
         }
       }
       ptx::tc_fence_before();

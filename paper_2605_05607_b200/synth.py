@@ -76,6 +76,18 @@ CONFIGS: Dict[str, MoEConfig] = {
                      bias="zipf", zipf_s=1.2, seed=1),
 }
 
+# The paper's own evaluation shapes (Table "Model Configurations": Small / Medium / Large, the
+# Large one being DeepSeek-V3's; top-k candidates 8 / 16 / 32), one GPU's share of a 32-GPU
+# expert-parallel group: G = 32 logical groups, T = 4 sequences of the table's length, sigmoid
+# scores as in the DeepSeek-V3 router.  The table gives no batch size: T is this build's choice.
+_PAPER_SIZES = {"S": dict(T=4 * 2048, d=2048, f=512, E=64), "M": dict(T=4 * 4096, d=4096, f=1024, E=128),
+                "L": dict(T=4 * 8192, d=7168, f=2048, E=256)}
+PAPER_CONFIGS: Dict[str, MoEConfig] = {
+    f"{size}{k}": MoEConfig(f"{size}{k}", k=k, G=32, score_fn=SCORE_SIGMOID, **dims)
+    for size, dims in _PAPER_SIZES.items() for k in (8, 16, 32)
+}
+ALL_CONFIGS: Dict[str, MoEConfig] = {**CONFIGS, **PAPER_CONFIGS}
+
 _TID = {"x": 1, "w_gate": 2, "w1": 3, "w3": 4, "w2": 5, "perm": 6, "fav": 7}
 
 

@@ -23,9 +23,11 @@ class Slabs:
         return synth.bf16_bits(self.w[int(e)])
 
 
-@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5a", "C5b"])
+# C2..C5b: the benchmark configurations; S32 / M16: two of the paper's own evaluation shapes
+# (Small at top-32 of 64 experts, Medium at top-16), 32 groups
+@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5a", "C5b", "S32", "M16"])
 def test_fullsize_layer(name):
-    cfg = synth.CONFIGS[name]
+    cfg = synth.ALL_CONFIGS[name]
     run = H.Run(cfg)
     lay_dev = B.alloc_layout(run.shape)
     run.layer(logits=run.logits, topk_idx=run.idx, topk_w=run.w, layout=lay_dev)
