@@ -13,70 +13,60 @@
 // producers.  Accumulators are double-buffered in TMEM (2 x 256 columns): the epilogue of tile i
 // overlaps the main loop of tile i+1.  Every wait is bounded.
 //
+// Pipeline: 4 stages, each an A tile (16 KiB, gathered) and a B tile (32 KiB, TMA) behind one
+// full / one empty barrier.  The gather threads never wait for their own copies: after issuing the
+// cp.async copies of a stage each thread posts cp.async.mbarrier.arrive.noinc on the stage's full
+// barrier, so the barrier completes exactly when the last row has landed (and the TMA bytes are
+// in), independent of how far the issuing threads have moved on.  An earlier form published a
+// stage only when the copies of two later stages had been issued (commit groups, wait, proxy
+// fence, arrive): the publication then trailed the tensor pipe by one stage and the kernel ran
+// 8-11 % (K = 4096) to 30 % (K = 7168, rows gathered from DRAM) slower; deeper or split A / B
+// rings on that form recovered only part of it and cost a second wait per k-block.
+//
 // A CTA-pair (cta_group::2) variant of this kernel was measured slower: with the UMMA twice as
-// fast per CTA the gather -> fence -> arrive -> UMMA chain of the peer CTA no longer fits the
-// pipeline depth, and TMA tile::gather4 sustains only one 4-row instruction per ~40 ns.
+// fast per CTA the gather -> arrive -> UMMA chain of the peer CTA no longer fits the pipeline
+// depth, and TMA tile::gather4 sustains only one 4-row instruction per ~40 ns.
 #include "ffn_common.cuh"
 
 namespace tcmoe {
 namespace ffn {
 namespace {
 
-// Two pipeline shapes (template parameter SPLIT), chosen by the host from K:
-//  - joint (SPLIT = false): 4 stages, each holding an A and a B tile behind one full / one empty
-//    barrier; the UMMA thread does one wait and one commit per k-block.  Best for K <= 4096
-//    (Mixtral-, GPT-OSS-, Qwen3-shaped layers: +6..9 % over the split form, measured sustained).
-//  - split (SPLIT = true): the gathered A tile has a ring of its own, one stage and one cp.async
-//    group deeper (5 x 16 KiB, lag 3), the weights keep 4 x 32 KiB; two waits and two commits per
-//    k-block.  Best for long K with rows gathered from DRAM (DeepSeek-V3-shaped, K = 7168: GEMM-1
-//    +10 %, whole FFN +14 % sustained, same box, alternating runs).
-constexpr int NB = 4;                        // B stages
+constexpr int NSTAGE = 4;
 constexpr int A_BYTES = BM * BK * 2;         // 16 KiB
 constexpr int B_BYTES = UMMA_N * BK * 2;     // 32 KiB = four 64-column slabs of 8 KiB
-constexpr int NA_MAX = 5;
-constexpr int NUM_BARS = 2 * NA_MAX + 2 * NB + 4;
-constexpr int SMEM_BYTES = 1024 + NA_MAX * A_BYTES + NB * B_BYTES + NUM_BARS * 8 + 64 + 2 * (MAX_E + 1) * 4;
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int NUM_BARS = 2 * NSTAGE + 4;
+constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + 2 * (MAX_E + 1) * 4;
 constexpr int THREADS = 320;
+constexpr int GATHER_THREADS = 128;
 constexpr int BN_OUT = 128;
 constexpr uint32_t IDESC = idesc_bf16(BM);
 
-template <bool SPLIT>
 __global__ void __launch_bounds__(THREADS, 1)
 ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w3,
                  const GemmParams p) {
-  constexpr int NA = SPLIT ? 5 : 4;            // A stages
-  constexpr int GATHER_LAG = SPLIT ? 3 : 2;    // cp.async groups kept in flight per gather thread
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + NA_MAX * A_BYTES + NB * B_BYTES);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + NSTAGE * STAGE_BYTES);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + NUM_BARS);
   int* abort_s = reinterpret_cast<int*>(tmem_slot + 1);
   int* tp_s = reinterpret_cast<int*>(tmem_slot + 16);
   int* eoff_s = tp_s + (MAX_E + 1);
 
-  const uint32_t a_ring = ptx::smem_u32(smem);
-  const uint32_t b_ring = a_ring + NA_MAX * A_BYTES;
+  const uint32_t smem_base = ptx::smem_u32(smem);
   const uint32_t bar_base = ptx::smem_u32(bars);
-  // joint form: the B barriers are the A barriers (NA == NB)
-  auto afull_bar = [&](int s) { return bar_base + 8u * s; };
-  auto aempty_bar = [&](int s) { return bar_base + 8u * (NA_MAX + s); };
-  auto bfull_bar = [&](int s) { return SPLIT ? bar_base + 8u * (2 * NA_MAX + s) : afull_bar(s); };
-  auto bempty_bar = [&](int s) { return SPLIT ? bar_base + 8u * (2 * NA_MAX + NB + s) : aempty_bar(s); };
-  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * NA_MAX + 2 * NB + b); };
-  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * NA_MAX + 2 * NB + 2 + b); };
+  auto full_bar = [&](int s) { return bar_base + 8u * s; };
+  auto empty_bar = [&](int s) { return bar_base + 8u * (NSTAGE + s); };
+  auto tfull_bar = [&](int b) { return bar_base + 8u * (2 * NSTAGE + b); };
+  auto tempty_bar = [&](int b) { return bar_base + 8u * (2 * NSTAGE + 2 + b); };
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < NA; ++s) {
-      ptx::mbar_init(afull_bar(s), SPLIT ? 4 : 5);   // one lane per gather warp (+ the TMA thread when joint)
-      ptx::mbar_init(aempty_bar(s), 1);              // tcgen05.commit
-    }
-    if (SPLIT) {
-      for (int s = 0; s < NB; ++s) {
-        ptx::mbar_init(bfull_bar(s), 1);    // TMA thread (expect_tx)
-        ptx::mbar_init(bempty_bar(s), 1);   // tcgen05.commit
-      }
+    for (int s = 0; s < NSTAGE; ++s) {
+      ptx::mbar_init(full_bar(s), GATHER_THREADS + 1);   // every gather thread's copies + the TMA thread (expect_tx)
+      ptx::mbar_init(empty_bar(s), 1);                   // tcgen05.commit
     }
     for (int b = 0; b < 2; ++b) {
       ptx::mbar_init(tfull_bar(b), 1);      // tcgen05.commit
@@ -161,17 +151,17 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
         const Tile t = tile_of(w);
         bool ok = true;
         for (int kb = 0; kb < KB; ++kb, ++it) {
-          const int s = it % NB;
-          if (!ptx::mbar_wait(bempty_bar(s), ((it / NB) & 1) ^ 1, abort_flag, global_abort)) {
+          const int s = it % NSTAGE;
+          if (!ptx::mbar_wait(empty_bar(s), ((it / NSTAGE) & 1) ^ 1, abort_flag, global_abort)) {
             timeout(2); ok = false; break;
           }
-          const uint32_t sb = b_ring + s * B_BYTES;
-          ptx::mbar_arrive_expect_tx(bfull_bar(s), B_BYTES);
+          const uint32_t sb = smem_base + s * STAGE_BYTES + A_BYTES;
+          ptx::mbar_arrive_expect_tx(full_bar(s), B_BYTES);
           const int k0 = kb * BK;
-          ptx::tma_load_3d(sb, &map_w1, bfull_bar(s), t.n0, k0, t.e);
-          ptx::tma_load_3d(sb + 8192, &map_w1, bfull_bar(s), t.n0 + 64, k0, t.e);
-          ptx::tma_load_3d(sb + 16384, &map_w3, bfull_bar(s), t.n0, k0, t.e);
-          ptx::tma_load_3d(sb + 24576, &map_w3, bfull_bar(s), t.n0 + 64, k0, t.e);
+          ptx::tma_load_3d(sb, &map_w1, full_bar(s), t.n0, k0, t.e);
+          ptx::tma_load_3d(sb + 8192, &map_w1, full_bar(s), t.n0 + 64, k0, t.e);
+          ptx::tma_load_3d(sb + 16384, &map_w3, full_bar(s), t.n0, k0, t.e);
+          ptx::tma_load_3d(sb + 24576, &map_w3, full_bar(s), t.n0 + 64, k0, t.e);
         }
         if (!ok) break;
       }
@@ -190,19 +180,17 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * UMMA_N);
         bool ok = true;
         for (int kb = 0; kb < KB; ++kb, ++it) {
-          const int sa_i = it % NA, sb_i = it % NB;
-          if (!ptx::mbar_wait(afull_bar(sa_i), (it / NA) & 1, abort_flag, global_abort) ||
-              (SPLIT && !ptx::mbar_wait(bfull_bar(sb_i), (it / NB) & 1, abort_flag, global_abort))) {
+          const int s = it % NSTAGE;
+          if (!ptx::mbar_wait(full_bar(s), (it / NSTAGE) & 1, abort_flag, global_abort)) {
             timeout(4); ok = false; break;
           }
           ptx::tc_fence_after();
-          const uint32_t sa = a_ring + sa_i * A_BYTES, sb = b_ring + sb_i * B_BYTES;
+          const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
           const uint64_t ad = desc_at(a_base, sa), bd = desc_at(b_base, sb);
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k)  // K = 16 per UMMA: A +32 B inside the swizzle row, B +2 atoms
             ptx::umma_bf16(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), IDESC, (kb | k) != 0);
-          ptx::umma_commit(aempty_bar(sa_i));   // free the stage(s) when these UMMAs have read them
-          if (SPLIT) ptx::umma_commit(bempty_bar(sb_i));
+          ptx::umma_commit(empty_bar(s));   // free the stage when these UMMAs have read it
         }
         if (!ok) break;
         ptx::umma_commit(tfull_bar(buf));   // accumulator complete
@@ -231,11 +219,11 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
       }
       bool ok = true;
       for (int kb = 0; kb < KB; ++kb, ++it) {
-        const int s = it % NA;
-        if (!ptx::mbar_wait(aempty_bar(s), ((it / NA) & 1) ^ 1, abort_flag, global_abort)) {
+        const int s = it % NSTAGE;
+        if (!ptx::mbar_wait(empty_bar(s), ((it / NSTAGE) & 1) ^ 1, abort_flag, global_abort)) {
           timeout(5); ok = false; break;
         }
-        const uint32_t sa = a_ring + s * A_BYTES;
+        const uint32_t sa = smem_base + s * STAGE_BYTES;
         const int col = kb * BK + chunk * 8;
         const bool kin = col < p.K;
 #pragma unroll
@@ -245,23 +233,13 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
           const bool on = kin && ((live >> j) & 1u);
           ptx::cp_async_16(dst, on ? (const void*)(src[j] + col) : (const void*)p.a_src, on ? 16u : 0u);
         }
-        ptx::cp_async_commit();
-        if (it >= GATHER_LAG) {
-          ptx::cp_async_wait<GATHER_LAG>();
-          ptx::fence_proxy_async_smem();
-          __syncwarp();
-          if (lane == 0) ptx::mbar_arrive(afull_bar((it - GATHER_LAG) % NA));
-        }
+        // one arrival on the stage's full barrier once the copies above have landed; the thread
+        // itself goes straight on to the next stage
+        ptx::cp_async_arrive_noinc(full_bar(s));
       }
       if (!ok) break;
     }
-    ptx::cp_async_wait<0>();
-    ptx::fence_proxy_async_smem();
-    __syncwarp();
-    if (lane == 0) {
-      const uint32_t first = it >= GATHER_LAG ? it - GATHER_LAG : 0;
-      for (uint32_t i = first; i < it; ++i) ptx::mbar_arrive(afull_bar(i % NA));
-    }
+    ptx::cp_async_wait_all();   // nothing may still be in flight towards shared memory at exit
   }
 
   ptx::tc_fence_before();
@@ -283,16 +261,12 @@ cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUt
   static bool attr_set[MAX_DEVICES] = {};   // the attribute is per device
   const int dev = current_device();
   if (!attr_set[dev]) {
-    cudaError_t e =
-        cudaFuncSetAttribute(ffn_gemm1_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(ffn_gemm1_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
   }
   ProfileScope prof(KID_GEMM1, st);
-  if (p.K >= 6144) return launch_pdl(ffn_gemm1_kernel<true>, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);
-  return launch_pdl(ffn_gemm1_kernel<false>, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);
+  return launch_pdl(ffn_gemm1_kernel, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);
 }
 
 }  // namespace ffn
