@@ -188,7 +188,11 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
       }
       ptx::tc_fence_before();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(buf), 0));
+      // "accumulator buffer drained": the tcgen05.ld results are in registers (wait::ld above), so a
+      // relaxed arrival is enough; a releasing one would first wait for this warp's row stores to
+      // become visible cluster-wide, which on short-K tiles stalls the next-but-one main loop
+      // (K = 512: 860 -> 1049 TFLOP/s with the relaxed form)
+      if (lane == 0) ptx::mbar_arrive_cluster_relaxed(ptx::mapa(tempty_bar(buf), 0));
     }
   } else if (warp == 4) {
     // ================================ TMA producer (both CTAs) ================================
