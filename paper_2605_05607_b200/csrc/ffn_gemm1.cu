@@ -37,7 +37,9 @@ constexpr int A_BYTES = BM * BK * 2;         // 16 KiB
 constexpr int B_BYTES = UMMA_N * BK * 2;     // 32 KiB = four 64-column slabs of 8 KiB
 constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int NUM_BARS = 2 * NSTAGE + 4;
-constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + 2 * (MAX_E + 1) * 4;
+constexpr int STAGE_OUT_WARP = 32 * 144;     // epilogue transpose buffer of one warp: 32 rows x (128 + 16) bytes
+constexpr int TABLE_BYTES = (2 * (MAX_E + 1) * 4 + 15) & ~15;
+constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + TABLE_BYTES + 4 * STAGE_OUT_WARP;
 constexpr int THREADS = 320;
 constexpr int GATHER_THREADS = 128;
 constexpr int BN_OUT = 128;
@@ -53,6 +55,7 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
   int* abort_s = reinterpret_cast<int*>(tmem_slot + 1);
   int* tp_s = reinterpret_cast<int*>(tmem_slot + 16);
   int* eoff_s = tp_s + (MAX_E + 1);
+  const uint32_t stage_base = ptx::smem_u32(tp_s) + TABLE_BYTES;   // 16-byte aligned
 
   const uint32_t smem_base = ptx::smem_u32(smem);
   const uint32_t bar_base = ptx::smem_u32(bars);
@@ -112,31 +115,44 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
       const int buf = tl & 1;
       if (!ptx::mbar_wait_warp<true>(tfull_bar(buf), (tl >> 1) & 1, abort_flag, global_abort)) { timeout(1); break; }
       ptx::tc_fence_after();
-      const int lrow = warp * 32 + lane;
-      const bool valid = lrow < t.rows;
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UMMA_N);
-      __nv_bfloat16* orow = p.out + (size_t)(valid ? t.row0 + lrow : 0) * (size_t)p.out_ld + t.n0;
+      // A thread owns one accumulator row; 32 threads storing 16 bytes each to 32 different rows
+      // would cost 32 memory transactions per instruction.  The warp transposes 64 output columns
+      // at a time through shared memory (rows padded to 144 bytes: conflict-free both ways) and
+      // stores whole 128-byte row segments, 8 lanes per row, 4 rows per instruction.
+      const uint32_t stage = stage_base + (uint32_t)(warp * STAGE_OUT_WARP);
+      const int srow = lane >> 3, piece = lane & 7;
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         uint32_t a1[32], a3[32];
         ptx::tmem_ld32(taddr + c * 32, a1);
         ptx::tmem_ld32(taddr + 128 + c * 32, a3);
         ptx::tmem_ld_wait();
-        if (valid) {
 #pragma unroll
-          for (int v = 0; v < 4; ++v) {
-            if (t.n0 + c * 32 + v * 8 < p.N) {
-              uint4 q;
-              uint32_t* qq = reinterpret_cast<uint32_t*>(&q);
+        for (int v = 0; v < 4; ++v) {
+          uint32_t q[4];
 #pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const int j = v * 8 + 2 * i;
-                qq[i] = pack2(silu_mul(__uint_as_float(a1[j]), __uint_as_float(a3[j])),
-                              silu_mul(__uint_as_float(a1[j + 1]), __uint_as_float(a3[j + 1])));
+          for (int i = 0; i < 4; ++i) {
+            const int j = v * 8 + 2 * i;
+            q[i] = pack2(silu_mul(__uint_as_float(a1[j]), __uint_as_float(a3[j])),
+                         silu_mul(__uint_as_float(a1[j + 1]), __uint_as_float(a3[j + 1])));
+          }
+          ptx::st_shared_v4(stage + lane * 144 + (c & 1) * 64 + v * 16, q[0], q[1], q[2], q[3]);
+        }
+        if (c & 1) {
+          __syncwarp();
+          const int col = t.n0 + (c - 1) * 32 + piece * 8;
+          if (col < p.N) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int r = i * 4 + srow;           // row of this warp's 32
+              if (warp * 32 + r < t.rows) {
+                const uint4 q = ptx::ld_shared_v4(stage + r * 144 + piece * 16);
+                *reinterpret_cast<uint4*>(p.out + (size_t)(t.row0 + warp * 32 + r) * (size_t)p.out_ld + col) = q;
               }
-              *reinterpret_cast<uint4*>(orow + c * 32 + v * 8) = q;
             }
           }
+          __syncwarp();
         }
       }
       ptx::tc_fence_before();
