@@ -32,7 +32,7 @@ KERNELS_PER_STEP = 10  # gate split, gate, topk, masks, scan, offsets, fill, gem
 
 # DRAM bytes (read + write) of one GEMM-1 launch from ncu captures summarised under profiles/;
 # None until a capture of that workload exists.
-GEMM1_DRAM_TRAFFIC = {"C2": 1.944110e9 + 228.062e6}   # profiles/ffn_gemm_C2_ncu_full.md
+GEMM1_DRAM_TRAFFIC = {"C2": 1.960784e9 + 229.266e6}   # profiles/ffn_gemm_C2_ncu_full.md
 
 
 def peaks():
