@@ -171,6 +171,33 @@ int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, co
                    const void* w1, const void* w3, const void* w2, void* y_dev, void* y_host,
                    void* ws, size_t ws_bytes, void* stream);
 
+/* ---- FP8 form of the expert FFN --------------------------------------------------------------
+ * Sec. VI-A evaluates the DeepSeek-V3 experts with FP8 GEMM kernels and gives no recipe; this
+ * library's reading: E4M3 elements (largest finite value 448, round to nearest even, saturating),
+ * one fp32 scale per activation row and one per (expert, output column) of a weight matrix,
+ * scale = fl32(max|v| / 448) (1 for an all-zero vector), code = e4m3(fl32(v / scale)); fp32
+ * accumulation; the scales multiply the accumulator in the epilogue; h is written as bf16 and
+ * quantised per row before GEMM-2. */
+
+/* src bf16 [rows, cols] -> dst E4M3 codes [rows, cols] (one byte each), scale fp32 [rows].
+ * cols % 8 == 0; src 16-byte, dst 8-byte aligned.  Device pointers; enqueues on `stream`. */
+int moe_quantize_rows(const void* src, int64_t rows, int64_t cols, void* dst, float* scale, void* stream);
+
+/* w bf16 [E, K, N] (N contiguous, the layout moe_expert_ffn takes) -> wq E4M3 codes [E, N, K]
+ * (K contiguous: the K-major operand of the FP8 GEMMs), scale fp32 [E, N].  A one-time
+ * preparation of static weights. */
+int moe_quantize_weights(const void* w, int32_t E, int32_t K, int32_t N, void* wq, float* scale, void* stream);
+
+/* moe_expert_ffn on quantised operands: xq E4M3 [rows of the dispatched buffer, d] with row
+ * scales sx (row r of expert e reads dispatched row layout->row_src[r]); w1q, w3q [E, f, d] with
+ * s1, s3 [E, f]; w2q [E, d, f] with s2 [E, d] (all from moe_quantize_weights).  o bf16 [T*k, d] as
+ * in moe_expert_ffn (gate weight in the epilogue unless MOE_FLAG_WEIGHT_IN_COMBINE).  Needs
+ * d % 16 == 0 and f % 16 == 0 (MOE_ERR_UNSUPPORTED_SHAPE otherwise); the workspace holds h (bf16),
+ * its E4M3 copy and its row scales. */
+int moe_expert_ffn_fp8(const moe_shape_t* shape, const void* xq, const float* sx, const moe_layout_t* layout,
+                       const float* topk_w, const void* w1q, const float* s1, const void* w3q, const float* s3,
+                       const void* w2q, const float* s2, void* o, void* ws, size_t ws_bytes, void* stream);
+
 /* Dispatch without a workspace (the paper has no counterpart; this entry point exists for
  * callers that cannot supply scratch memory).  Some users of this library run where device
  * memory cannot be obtained around the call: plugins that execute inside a host framework's

@@ -35,7 +35,8 @@ MOE_FLAG_COMBINE_IN_EPILOGUE = 2
 
 EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "moe_status", "moe_strerror",
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",
-           "moe_profile_enable", "moe_profile_read", "moe_dispatch_noalloc")
+           "moe_profile_enable", "moe_profile_read", "moe_dispatch_noalloc", "moe_quantize_rows",
+           "moe_quantize_weights", "moe_expert_ffn_fp8")
 
 
 class MoEShape(ctypes.Structure):
@@ -80,6 +81,9 @@ def lib() -> ctypes.CDLL:
         L.moe_layer.argtypes = [shp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, lay, vp, sz, vp]
         L.moe_layer_host.argtypes = [shp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, sz, vp]
         L.moe_dispatch_noalloc.argtypes = [shp, vp, vp, lay, vp, vp, vp]
+        L.moe_quantize_rows.argtypes = [vp, i64, i64, vp, vp, vp]
+        L.moe_quantize_weights.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
+        L.moe_expert_ffn_fp8.argtypes = [shp, vp, vp, lay, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.moe_profile_enable.argtypes = [ctypes.c_int]
         L.moe_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
         for name in EXPORTS:
@@ -194,6 +198,28 @@ def moe_expert_ffn(shape, xg, layout: Layout, topk_w, w1, w3, w2, o, ws, stream=
     _check("moe_expert_ffn", lib().moe_expert_ffn(ctypes.byref(shape), _ptr(xg), ctypes.byref(c), _ptr(topk_w),
                                                   _ptr(w1), _ptr(w3), _ptr(w2), _ptr(o), _ptr(ws), ws.numel(),
                                                   _stream(stream)))
+
+
+def moe_quantize_rows(src, dst, scale, stream=None) -> None:
+    """src bf16 [rows, cols] -> dst uint8 [rows, cols] (E4M3 codes), scale fp32 [rows]."""
+    rows, cols = src.shape
+    _check("moe_quantize_rows", lib().moe_quantize_rows(_ptr(src), ctypes.c_int64(rows), ctypes.c_int64(cols),
+                                                        _ptr(dst), _ptr(scale), _stream(stream)))
+
+
+def moe_quantize_weights(w, wq, scale, stream=None) -> None:
+    """w bf16 [E, K, N] -> wq uint8 [E, N, K] (E4M3 codes, K contiguous), scale fp32 [E, N]."""
+    E, K, N = w.shape
+    _check("moe_quantize_weights", lib().moe_quantize_weights(_ptr(w), E, K, N, _ptr(wq), _ptr(scale),
+                                                              _stream(stream)))
+
+
+def moe_expert_ffn_fp8(shape, xq, sx, layout: Layout, topk_w, w1q, s1, w3q, s3, w2q, s2, o, ws, stream=None) -> None:
+    c = layout.c()
+    _check("moe_expert_ffn_fp8", lib().moe_expert_ffn_fp8(ctypes.byref(shape), _ptr(xq), _ptr(sx), ctypes.byref(c),
+                                                          _ptr(topk_w), _ptr(w1q), _ptr(s1), _ptr(w3q), _ptr(s3),
+                                                          _ptr(w2q), _ptr(s2), _ptr(o), _ptr(ws), ws.numel(),
+                                                          _stream(stream)))
 
 
 def moe_combine(shape, o, layout: Layout, topk_idx, topk_w, pg, y, ws, stream=None) -> None:

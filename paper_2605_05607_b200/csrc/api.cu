@@ -14,7 +14,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Regions of the workspace, in order.  Every region starts on a 1 KiB boundary.
 struct WsPlan {
-  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, wsplit, h, o, logits, topk_idx, topk_w;
+  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, wsplit, h, hq, sh, o, logits, topk_idx, topk_w;
   size_t expert_counts, expert_offsets, group_counts, group_offsets, pair_row, row_pair, al, disp_token, row_src;
   size_t total;
   int W;
@@ -44,6 +44,8 @@ WsPlan plan(const moe_shape_t& s) {
   p.mp_prefix = take((E + 1) * 4);
   p.wsplit = take(gate_split_bytes(s.d, s.E));
   p.h = take(P * (size_t)s.f * 2);
+  p.hq = take(P * (size_t)s.f);   // FP8 form: E4M3 copy of h and its row scales
+  p.sh = take(P * 4);
   // o [P, d] bf16, or the fp32 token accumulators [T, d] of the Combine-in-epilogue form
   p.o = take((P * 2 > T * 4 ? P * 2 : T * 4) * (size_t)s.d);
   p.logits = take(T * E * 4);
@@ -309,6 +311,67 @@ int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t*
   TCMOE_CUDA(launch_tile_prefix(to_shape(*shape), layout->expert_counts, at<int32_t>(ws, p.mt_prefix),
                                 at<int32_t>(ws, p.mp_prefix), static_cast<cudaStream_t>(stream)));
   TCMOE_CUDA(launch_expert_ffn(to_shape(*shape), a, static_cast<cudaStream_t>(stream)));
+  return MOE_OK;
+}
+
+int moe_quantize_rows(const void* src, int64_t rows, int64_t cols, void* dst, float* scale, void* stream) {
+  if (rows < 0 || cols <= 0 || cols > (1ll << 30)) return MOE_ERR_INVALID_ARG;
+  if (cols % 8 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
+  if (rows > 0 && (src == nullptr || dst == nullptr || scale == nullptr)) return MOE_ERR_INVALID_ARG;
+  if (!aligned(src, 16) || !aligned(dst, 8) || !aligned(scale, 4)) return MOE_ERR_MISALIGNED;
+  if (!have_device()) return MOE_ERR_CUDA;
+  TCMOE_CUDA(launch_quantize_rows(src, rows, (int)cols, dst, scale, static_cast<cudaStream_t>(stream)));
+  return MOE_OK;
+}
+
+int moe_quantize_weights(const void* w, int32_t E, int32_t K, int32_t N, void* wq, float* scale, void* stream) {
+  if (E <= 0 || K <= 0 || N <= 0 || E > 65535) return MOE_ERR_INVALID_ARG;
+  if (w == nullptr || wq == nullptr || scale == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!aligned(w, 16) || !aligned(wq, 16) || !aligned(scale, 4)) return MOE_ERR_MISALIGNED;
+  if (!have_device()) return MOE_ERR_CUDA;
+  TCMOE_CUDA(launch_quantize_weights(w, E, K, N, wq, scale, static_cast<cudaStream_t>(stream)));
+  return MOE_OK;
+}
+
+int moe_expert_ffn_fp8(const moe_shape_t* shape, const void* xq, const float* sx, const moe_layout_t* layout,
+                       const float* topk_w, const void* w1q, const float* s1, const void* w3q, const float* s3,
+                       const void* w2q, const float* s2, void* o, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (shape->d % 16 != 0 || shape->f % 16 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;   // 16-byte rows of 8-bit elements
+  if (xq == nullptr || sx == nullptr || w1q == nullptr || w3q == nullptr || w2q == nullptr || s1 == nullptr ||
+      s3 == nullptr || s2 == nullptr || o == nullptr)
+    return MOE_ERR_INVALID_ARG;
+  if (shape->flags & MOE_FLAG_COMBINE_IN_EPILOGUE) return MOE_ERR_INVALID_ARG;
+  const bool in_combine = (shape->flags & MOE_FLAG_WEIGHT_IN_COMBINE) != 0;
+  if (!in_combine && topk_w == nullptr) return MOE_ERR_INVALID_ARG;
+  if ((rc = check_layout(layout)) != MOE_OK) return rc;
+  if (!aligned(xq, 128) || !aligned(w1q, 128) || !aligned(w3q, 128) || !aligned(w2q, 128) || !aligned(o, 128) ||
+      !aligned(topk_w, 16) || !aligned(sx, 4) || !aligned(s1, 4) || !aligned(s3, 4) || !aligned(s2, 4))
+    return MOE_ERR_MISALIGNED;
+  WsPlan p;
+  if ((rc = check_ws(shape, ws, ws_bytes, &p)) != MOE_OK) return rc;
+  if (!have_device()) return MOE_ERR_CUDA;
+  FfnArgs a{};
+  a.a_src = xq;
+  a.gather_idx = layout->row_src;
+  a.gather_div = 1;
+  a.w1 = w1q;
+  a.w3 = w3q;
+  a.w2 = w2q;
+  a.h = at<void>(ws, p.h);
+  a.o = o;
+  a.topk_w = in_combine ? nullptr : topk_w;
+  a.row_pair = layout->row_pair;
+  a.expert_offsets = layout->expert_offsets;
+  a.mt_prefix = at<int32_t>(ws, p.mt_prefix);
+  a.mp_prefix = at<int32_t>(ws, p.mp_prefix);
+  a.status = at<int32_t>(ws, p.status);
+  Fp8Args q{sx, s1, s3, s2, at<void>(ws, p.hq), at<float>(ws, p.sh)};
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  TCMOE_CUDA(launch_tile_prefix(to_shape(*shape), layout->expert_counts, at<int32_t>(ws, p.mt_prefix),
+                                at<int32_t>(ws, p.mp_prefix), st));
+  TCMOE_CUDA(launch_expert_ffn_fp8(to_shape(*shape), a, q, st));
   return MOE_OK;
 }
 

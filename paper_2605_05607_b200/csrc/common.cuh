@@ -104,6 +104,17 @@ struct FfnArgs {
   int32_t* status;
 };
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st);
+// FP8 form of the expert FFN: a.a_src / a.w1 / a.w3 / a.w2 hold E4M3 codes (weights [E, N, K]).
+struct Fp8Args {
+  const float* sx;            // per source row of a.a_src
+  const float *s1, *s3, *s2;  // per (expert, output column)
+  void* hq;                   // [P, f] E4M3 scratch
+  float* sh;                  // [P] scratch: row scales of h
+};
+cudaError_t launch_expert_ffn_fp8(const Shape& s, const FfnArgs& a, const Fp8Args& q, cudaStream_t st);
+// quant.cu: bf16 -> E4M3 with one scale per row / per (expert, output column)
+cudaError_t launch_quantize_rows(const void* src, long long rows, int cols, void* dst, float* scale, cudaStream_t st);
+cudaError_t launch_quantize_weights(const void* w, int E, int K, int N, void* wq, float* scale, cudaStream_t st);
 int sm_count();
 int current_device();   // index of the current CUDA device, clamped to [0, MAX_DEVICES)
 constexpr int MAX_DEVICES = 64;   // per-device caches (kernel attributes, SM counts) are arrays of this size

@@ -44,6 +44,32 @@ bool make_act_map(CUtensorMap* map, const void* base, int rows, int K) {
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// E4M3 weights [E, N, K] (K contiguous): box = 128 bytes of K x 128 output columns x 1, 128-byte swizzle
+bool make_weight_map_fp8(CUtensorMap* map, const void* base, int E, int N, int K) {
+  ffn::EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)N, (cuuint64_t)E};
+  cuuint64_t strides[2] = {(cuuint64_t)K, (cuuint64_t)N * K};
+  cuuint32_t box[3] = {128, 128, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// E4M3 activations [rows, K]: box = 128 bytes of K x 128 rows
+bool make_act_map_fp8(CUtensorMap* map, const void* base, int rows, int K) {
+  ffn::EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)K};
+  cuuint32_t box[2] = {128, ffn::BM};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 int current_device() {
@@ -89,7 +115,7 @@ cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st)
   g1.N = s.f;
   g1.n_tiles = (s.f + 127) / 128;
   g1.status = a.status;
-  cudaError_t err = ffn::launch_gemm1(g1, m_w1, m_w3, st);
+  cudaError_t err = ffn::launch_gemm1(g1, m_w1, m_w3, false, st);
   if (err != cudaSuccess) return err;
 
   ffn::GemmParams g2{};
@@ -106,7 +132,56 @@ cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st)
   g2.status = a.status;
   g2.y_acc = a.y_acc;
   g2.y_div = s.k;
-  return ffn::launch_gemm2(g2, m_w2, m_h, st);
+  return ffn::launch_gemm2(g2, m_w2, m_h, false, st);
+}
+
+// FP8 form: GEMM-1 on E4M3 rows and weights -> h (bf16) -> per-row quantisation of h -> GEMM-2 on E4M3.
+cudaError_t launch_expert_ffn_fp8(const Shape& s, const FfnArgs& a, const Fp8Args& q, cudaStream_t st) {
+  if (s.T == 0) return cudaSuccess;
+  const int P = s.T * s.k;
+  CUtensorMap m_w1, m_w3, m_w2, m_h;
+  if (!make_weight_map_fp8(&m_w1, a.w1, s.E, s.f, s.d) || !make_weight_map_fp8(&m_w3, a.w3, s.E, s.f, s.d) ||
+      !make_weight_map_fp8(&m_w2, a.w2, s.E, s.d, s.f) || !make_act_map_fp8(&m_h, q.hq, P, s.f))
+    return cudaErrorInvalidValue;
+
+  ffn::GemmParams g1{};
+  g1.a_src = a.a_src;
+  g1.a_ld = s.d;
+  g1.gather_idx = a.gather_idx;
+  g1.gather_div = a.gather_div;
+  g1.out = static_cast<__nv_bfloat16*>(a.h);
+  g1.out_ld = s.f;
+  g1.expert_offsets = a.expert_offsets;
+  g1.tile_prefix = a.mt_prefix;
+  g1.E = s.E;
+  g1.K = s.d;
+  g1.N = s.f;
+  g1.n_tiles = (s.f + 127) / 128;
+  g1.status = a.status;
+  g1.a_scale = q.sx;
+  g1.b_scale = q.s1;
+  g1.b_scale2 = q.s3;
+  cudaError_t err = ffn::launch_gemm1(g1, m_w1, m_w3, true, st);
+  if (err != cudaSuccess) return err;
+  if ((err = launch_quantize_rows(a.h, P, s.f, q.hq, q.sh, st)) != cudaSuccess) return err;
+
+  ffn::GemmParams g2{};
+  g2.out = static_cast<__nv_bfloat16*>(a.o);
+  g2.out_ld = s.d;
+  g2.topk_w = a.topk_w;
+  g2.row_pair = a.row_pair;
+  g2.expert_offsets = a.expert_offsets;
+  g2.tile_prefix = a.mp_prefix;
+  g2.E = s.E;
+  g2.K = s.f;
+  g2.N = s.d;
+  g2.n_tiles = (s.d + 255) / 256;
+  g2.status = a.status;
+  g2.y_acc = a.y_acc;
+  g2.y_div = s.k;
+  g2.a_scale = q.sh;
+  g2.b_scale = q.s2;
+  return ffn::launch_gemm2(g2, m_w2, m_h, true, st);
 }
 
 }  // namespace tcmoe

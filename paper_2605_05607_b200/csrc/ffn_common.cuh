@@ -16,8 +16,8 @@ constexpr int UMMA_N = 256;   // accumulator columns per tile
 constexpr int MAX_E = 1024;
 
 struct GemmParams {
-  const __nv_bfloat16* a_src;   // GEMM-1 gather source (xg or x)
-  int a_ld;
+  const void* a_src;            // GEMM-1 gather source (xg or x): bf16, or E4M3 codes in the FP8 form
+  int a_ld;                     // elements per source row
   const int32_t* gather_idx;    // row_src, or row_pair with gather_div = k (token = row_pair / k)
   int gather_div;
   __nv_bfloat16* out;
@@ -29,6 +29,11 @@ struct GemmParams {
                                 // 256-row CTA-pair tiles for GEMM-2)
   int E, K, N, n_tiles;
   int32_t* status;
+  // FP8 form only: per-row scale of the A operand (indexed like the A rows: gather source rows
+  // for GEMM-1, expert-sorted rows for GEMM-2) and per-(expert, output column) scales of B
+  const float* a_scale;
+  const float* b_scale;         // [E, N]   (GEMM-1: W1)
+  const float* b_scale2;        // [E, N]   (GEMM-1: W3)
   float* y_acc;                 // GEMM-2 with Combine in its epilogue: fp32 [T, N] accumulator, token
   int y_div;                    // of row r = row_pair[r] / y_div (NULL: rows go to `out`)
 };
@@ -79,6 +84,12 @@ __device__ __forceinline__ uint64_t desc_at(uint64_t base, uint32_t smem_addr) {
   return base | (uint64_t)((smem_addr & 0x3FFFF) >> 4);
 }
 
+// instruction descriptor of the FP8 form: D fp32, A/B E4M3 (format code 0), both K-major, N = 256, M = m
+__host__ __device__ constexpr uint32_t idesc_e4m3(int m) {
+  return (1u << 4) | (0u << 7) | (0u << 10) | (0u << 15) | (0u << 16) | ((uint32_t)(UMMA_N >> 3) << 17) |
+         ((uint32_t)(m >> 4) << 24);
+}
+
 // instruction descriptor: D fp32, A/B bf16, A K-major, B MN-major, N = 256, M = m
 __host__ __device__ constexpr uint32_t idesc_bf16(int m) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((uint32_t)(UMMA_N >> 3) << 17) |
@@ -96,8 +107,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, cudaStream_t st);
-cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, cudaStream_t st);
+// fp8 = false: bf16 operands, weights [E, K, N] (B MN-major).  fp8 = true: E4M3 operands, weights
+// [E, N, K] (B K-major), 128 elements of K per pipeline stage, scales applied in the epilogue.
+cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, bool fp8,
+                         cudaStream_t st);
+cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, bool fp8,
+                         cudaStream_t st);
 
 }  // namespace ffn
 }  // namespace tcmoe

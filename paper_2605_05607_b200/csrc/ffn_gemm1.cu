@@ -44,7 +44,12 @@ constexpr int THREADS = 320;
 constexpr int GATHER_THREADS = 128;
 constexpr int BN_OUT = 128;
 constexpr uint32_t IDESC = idesc_bf16(BM);
+constexpr uint32_t IDESC_F8 = idesc_e4m3(BM);
 
+// FP8 = true: A rows and weights are E4M3 codes, a stage holds 128 elements of K (the same 128
+// bytes per row), W1 / W3 come K-major from [E, N, K] as two 128-row boxes, and the epilogue applies
+// a_scale[source row] * b_scale[e, n] before the SwiGLU; h is written as bf16 either way.
+template <bool FP8>
 __global__ void __launch_bounds__(THREADS, 1)
 ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w3,
                  const GemmParams p) {
@@ -96,7 +101,8 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int total = tp_s[p.E] * p.n_tiles;
-  const int KB = (p.K + BK - 1) / BK;
+  constexpr int BK_ELEMS = FP8 ? 2 * BK : BK;   // K elements per stage: 128 bytes per row either way
+  const int KB = (p.K + BK_ELEMS - 1) / BK_ELEMS;
   volatile int* abort_flag = abort_s;
   const volatile int* global_abort = p.status + ST_ABORT;
 
@@ -122,6 +128,18 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
       // stores whole 128-byte row segments, 8 lanes per row, 4 rows per instruction.
       const uint32_t stage = stage_base + (uint32_t)(warp * STAGE_OUT_WARP);
       const int srow = lane >> 3, piece = lane & 7;
+      float sa = 1.f;   // FP8: scale of this thread's row (the gather source row)
+      const float *s1 = nullptr, *s3 = nullptr;
+      if (FP8) {
+        const int lrow = warp * 32 + lane;
+        if (lrow < t.rows) {
+          int idx = __ldg(p.gather_idx + t.row0 + lrow);
+          if (p.gather_div > 1) idx /= p.gather_div;
+          sa = __ldg(p.a_scale + idx);
+        }
+        s1 = p.b_scale + (size_t)t.e * p.N + t.n0;
+        s3 = p.b_scale2 + (size_t)t.e * p.N + t.n0;
+      }
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         uint32_t a1[32], a3[32];
@@ -134,8 +152,17 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             const int j = v * 8 + 2 * i;
-            q[i] = pack2(silu_mul(__uint_as_float(a1[j]), __uint_as_float(a3[j])),
-                         silu_mul(__uint_as_float(a1[j + 1]), __uint_as_float(a3[j + 1])));
+            float u0 = __uint_as_float(a1[j]), u1 = __uint_as_float(a1[j + 1]);
+            float g0 = __uint_as_float(a3[j]), g1 = __uint_as_float(a3[j + 1]);
+            if (FP8) {
+              const int n = c * 32 + j;
+              const bool in0 = t.n0 + n < p.N, in1 = t.n0 + n + 1 < p.N;
+              u0 *= sa * (in0 ? __ldg(s1 + n) : 0.f);
+              g0 *= sa * (in0 ? __ldg(s3 + n) : 0.f);
+              u1 *= sa * (in1 ? __ldg(s1 + n + 1) : 0.f);
+              g1 *= sa * (in1 ? __ldg(s3 + n + 1) : 0.f);
+            }
+            q[i] = pack2(silu_mul(u0, g0), silu_mul(u1, g1));
           }
           ptx::st_shared_v4(stage + lane * 144 + (c & 1) * 64 + v * 16, q[0], q[1], q[2], q[3]);
         }
@@ -173,11 +200,16 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
           }
           const uint32_t sb = smem_base + s * STAGE_BYTES + A_BYTES;
           ptx::mbar_arrive_expect_tx(full_bar(s), B_BYTES);
-          const int k0 = kb * BK;
-          ptx::tma_load_3d(sb, &map_w1, full_bar(s), t.n0, k0, t.e);
-          ptx::tma_load_3d(sb + 8192, &map_w1, full_bar(s), t.n0 + 64, k0, t.e);
-          ptx::tma_load_3d(sb + 16384, &map_w3, full_bar(s), t.n0, k0, t.e);
-          ptx::tma_load_3d(sb + 24576, &map_w3, full_bar(s), t.n0 + 64, k0, t.e);
+          const int k0 = kb * BK_ELEMS;
+          if (FP8) {   // K-major boxes of 128 output columns x 128 bytes of K
+            ptx::tma_load_3d(sb, &map_w1, full_bar(s), k0, t.n0, t.e);
+            ptx::tma_load_3d(sb + 16384, &map_w3, full_bar(s), k0, t.n0, t.e);
+          } else {     // MN-major slabs of 64 output columns x 64 rows of K
+            ptx::tma_load_3d(sb, &map_w1, full_bar(s), t.n0, k0, t.e);
+            ptx::tma_load_3d(sb + 8192, &map_w1, full_bar(s), t.n0 + 64, k0, t.e);
+            ptx::tma_load_3d(sb + 16384, &map_w3, full_bar(s), t.n0, k0, t.e);
+            ptx::tma_load_3d(sb + 24576, &map_w3, full_bar(s), t.n0 + 64, k0, t.e);
+          }
         }
         if (!ok) break;
       }
@@ -186,7 +218,7 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
     // ================================ UMMA issuer ================================
     if (lane == 0) {
       const uint64_t a_base = desc_base(16, 1024);
-      const uint64_t b_base = desc_base(BK * 128, 1024);
+      const uint64_t b_base = FP8 ? desc_base(16, 1024) : desc_base(BK * 128, 1024);   // K-major : MN-major
       uint32_t it = 0;
       int tl = 0;
       for (int w = blockIdx.x; w < total && !*abort_flag; w += gridDim.x, ++tl) {
@@ -204,8 +236,10 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
           const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
           const uint64_t ad = desc_at(a_base, sa), bd = desc_at(b_base, sb);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)  // K = 16 per UMMA: A +32 B inside the swizzle row, B +2 atoms
-            ptx::umma_bf16(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), IDESC, (kb | k) != 0);
+          for (int k = 0; k < 4; ++k) {   // 32 bytes of K per UMMA (16 bf16 / 32 E4M3): +32 B inside the swizzle row
+            if (FP8) ptx::umma_f8(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), IDESC_F8, (kb | k) != 0);
+            else ptx::umma_bf16(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), IDESC, (kb | k) != 0);   // B: +2 atoms
+          }
           ptx::umma_commit(empty_bar(s));   // free the stage when these UMMAs have read it
         }
         if (!ok) break;
@@ -220,16 +254,18 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
     uint32_t it = 0;
     for (int w = blockIdx.x; w < total && !*abort_flag; w += gridDim.x) {
       const Tile t = tile_of(w);
-      const __nv_bfloat16* src[8];
+      constexpr int ELEM = FP8 ? 1 : 2;   // bytes per element of the source rows
+      const uint8_t* src[8];
+      const uint8_t* base = static_cast<const uint8_t*>(p.a_src);
       uint32_t live = 0;
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const int lr = rbase + 16 * j;
-        src[j] = p.a_src;
+        src[j] = base;
         if (lr < t.rows) {
           int idx = __ldg(p.gather_idx + t.row0 + lr);
           if (p.gather_div > 1) idx /= p.gather_div;
-          src[j] = p.a_src + (size_t)idx * p.a_ld;
+          src[j] = base + (size_t)idx * p.a_ld * ELEM;
           live |= 1u << j;
         }
       }
@@ -240,14 +276,14 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
           timeout(5); ok = false; break;
         }
         const uint32_t sa = smem_base + s * STAGE_BYTES;
-        const int col = kb * BK + chunk * 8;
-        const bool kin = col < p.K;
+        const int col = kb * 128 + chunk * 16;   // byte offset inside the source row
+        const bool kin = col < p.K * ELEM;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
           const int lr = rbase + 16 * j;
           const uint32_t dst = sa + lr * 128 + ((chunk ^ (lr & 7)) << 4);
           const bool on = kin && ((live >> j) & 1u);
-          ptx::cp_async_16(dst, on ? (const void*)(src[j] + col) : (const void*)p.a_src, on ? 16u : 0u);
+          ptx::cp_async_16(dst, on ? (const void*)(src[j] + col) : (const void*)base, on ? 16u : 0u);
         }
         // one arrival on the stage's full barrier once the copies above have landed; the thread
         // itself goes straight on to the next stage
@@ -273,16 +309,20 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
 
 }  // namespace
 
-cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, cudaStream_t st) {
+cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, bool fp8,
+                         cudaStream_t st) {
   static bool attr_set[MAX_DEVICES] = {};   // the attribute is per device
   const int dev = current_device();
   if (!attr_set[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(ffn_gemm1_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm1_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(ffn_gemm1_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
   }
   ProfileScope prof(KID_GEMM1, st);
-  return launch_pdl(ffn_gemm1_kernel, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);
+  if (fp8) return launch_pdl(ffn_gemm1_kernel<true>, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);
+  return launch_pdl(ffn_gemm1_kernel<false>, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);
 }
 
 }  // namespace ffn

@@ -35,12 +35,16 @@ constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + TAB
 constexpr int THREADS = 192;
 constexpr int BN_OUT = 256;
 constexpr uint32_t IDESC = idesc_bf16(2 * BM);
+constexpr uint32_t IDESC_F8 = idesc_e4m3(2 * BM);
 constexpr uint32_t HINT = 4000;   // try_wait suspend-time hint (ns), see ptx::mbar_try_wait
 
 // RED = false: rows go to o (bf16), Combine is a later pass.  RED = true: Combine happens here
 // (Sec. V: the fused pipeline reduces expert outputs as GEMM-2 produces them): each weighted row is
 // added into the fp32 accumulator row of its token with vector reductions; o is never written.
-template <bool RED>
+// FP8 = true: h rows and weights are E4M3 codes, a stage holds 128 elements of K (the same 128 bytes
+// per row), W2 comes K-major from [E, N, K] as one 128-row box per CTA, and the epilogue applies
+// a_scale[row] * b_scale[e, n] together with the gate weight.
+template <bool RED, bool FP8>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_h,
                  const GemmParams p) {
@@ -95,7 +99,8 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int total = tp_s[p.E] * p.n_tiles;
-  const int KB = (p.K + BK - 1) / BK;
+  constexpr int BK_ELEMS = FP8 ? 2 * BK : BK;   // K elements per stage: 128 bytes per row either way
+  const int KB = (p.K + BK_ELEMS - 1) / BK_ELEMS;
   volatile int* abort_flag = abort_s;
   const volatile int* global_abort = p.status + ST_ABORT;
 
@@ -123,14 +128,23 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
       if (valid) {
         const int pair = __ldg(p.row_pair + grow);
         if (p.topk_w != nullptr) wr = __ldg(p.topk_w + pair);
+        if (FP8) wr *= __ldg(p.a_scale + grow);   // row scale of h joins the gate weight
         if (RED) yrow = p.y_acc + (size_t)(pair / p.y_div) * (size_t)p.N + t.n0;
       }
+      const float* sb_col = FP8 ? p.b_scale + (size_t)t.e * p.N + t.n0 : nullptr;
       if (RED) {
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
           uint32_t acc[32];
           ptx::tmem_ld32(taddr + c * 32, acc);
           ptx::tmem_ld_wait();
+          if (FP8) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int n = c * 32 + j;
+              acc[j] = __float_as_uint(__uint_as_float(acc[j]) * (t.n0 + n < p.N ? __ldg(sb_col + n) : 0.f));
+            }
+          }
           if (valid) {
 #pragma unroll
             for (int v = 0; v < 4; ++v) {
@@ -158,6 +172,14 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
           ptx::tmem_ld32(taddr + cc * 64 + 32, acc1);
           ptx::tmem_ld_wait_on(acc0);
           ptx::tmem_ld_wait_on(acc1);
+          if (FP8) {   // per-output-column weight scales
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int n = cc * 64 + j;
+              acc0[j] = __float_as_uint(__uint_as_float(acc0[j]) * (t.n0 + n < p.N ? __ldg(sb_col + n) : 0.f));
+              acc1[j] = __float_as_uint(__uint_as_float(acc1[j]) * (t.n0 + n + 32 < p.N ? __ldg(sb_col + n + 32) : 0.f));
+            }
+          }
 #pragma unroll
           for (int v = 0; v < 4; ++v) {
             ptx::st_shared_v4(stage + lane * 144 + v * 16,
@@ -210,10 +232,14 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
           const uint32_t lead_full = ptx::mapa(full_bar(s), 0);
           // the leader announces the bytes of both CTAs; the peer's copies only complete them
           if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
-          const int k0 = kb * BK;
+          const int k0 = kb * BK_ELEMS;
           ptx::tma_load_2d_pair(sa, &map_h, lead_full, k0, t.row0);
-          ptx::tma_load_3d_pair(sb, &map_w2, lead_full, t.n0 + rank * 128, k0, t.e);
-          ptx::tma_load_3d_pair(sb + 8192, &map_w2, lead_full, t.n0 + rank * 128 + 64, k0, t.e);
+          if (FP8) {   // one K-major box: this CTA's 128 output columns x 128 bytes of K
+            ptx::tma_load_3d_pair(sb, &map_w2, lead_full, k0, t.n0 + rank * 128, t.e);
+          } else {     // two MN-major slabs of 64 output columns x 64 rows of K
+            ptx::tma_load_3d_pair(sb, &map_w2, lead_full, t.n0 + rank * 128, k0, t.e);
+            ptx::tma_load_3d_pair(sb + 8192, &map_w2, lead_full, t.n0 + rank * 128 + 64, k0, t.e);
+          }
         }
         if (!ok) break;
       }
@@ -222,7 +248,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
     // ================================ UMMA issuer (leader CTA only) ================================
     if (rank == 0 && lane == 0) {
       const uint64_t a_base = desc_base(16, 1024);
-      const uint64_t b_base = desc_base(BK * 128, 1024);
+      const uint64_t b_base = FP8 ? desc_base(16, 1024) : desc_base(BK * 128, 1024);   // K-major : MN-major
       uint32_t it = 0;
       int tl = 0;
       for (int w = cluster_id; w < total && !*abort_flag; w += num_clusters, ++tl) {
@@ -242,8 +268,10 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
           const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
           const uint64_t ad = desc_at(a_base, sa), bd = desc_at(b_base, sb);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)  // K = 16 per UMMA: A +32 B inside the swizzle row, B +2 atoms
-            ptx::umma_bf16_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), IDESC, (kb | k) != 0);
+          for (int k = 0; k < 4; ++k) {   // 32 bytes of K per UMMA (16 bf16 / 32 E4M3): +32 B inside the swizzle row
+            if (FP8) ptx::umma_f8_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), IDESC_F8, (kb | k) != 0);
+            else ptx::umma_bf16_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), IDESC, (kb | k) != 0);   // B: +2 atoms
+          }
           // free the stage in both CTAs once these UMMAs have read it
           ptx::umma_commit_pair(ptx::mapa(empty_bar(s), 0));
           ptx::umma_commit_pair(ptx::mapa(empty_bar(s), 1));
@@ -285,7 +313,7 @@ int pair_grid() {
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    if (cudaOccupancyMaxActiveClusters(&clusters, ffn_gemm2_kernel<false>, &cfg) != cudaSuccess || clusters <= 0) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, ffn_gemm2_kernel<false, false>, &cfg) != cudaSuccess || clusters <= 0) {
       (void)cudaGetLastError();
       clusters = sm_count() / 2;
     }
@@ -296,19 +324,27 @@ int pair_grid() {
 
 }  // namespace
 
-cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, cudaStream_t st) {
+cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, bool fp8,
+                         cudaStream_t st) {
   static bool attr_set[MAX_DEVICES] = {};   // the attribute is per device
   const int dev = current_device();
   if (!attr_set[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(ffn_gemm2_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, true>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, true>, attr, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set[dev] = true;
   }
   ProfileScope prof(KID_GEMM2, st);
-  if (p.y_acc != nullptr) return launch_pdl(ffn_gemm2_kernel<true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
-  return launch_pdl(ffn_gemm2_kernel<false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
+  const bool red = p.y_acc != nullptr;
+  if (fp8) {
+    if (red) return launch_pdl(ffn_gemm2_kernel<true, true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
+    return launch_pdl(ffn_gemm2_kernel<false, true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
+  }
+  if (red) return launch_pdl(ffn_gemm2_kernel<true, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
+  return launch_pdl(ffn_gemm2_kernel<false, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
 }
 
 }  // namespace ffn
