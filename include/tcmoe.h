@@ -198,6 +198,15 @@ int moe_expert_ffn_fp8(const moe_shape_t* shape, const void* xq, const float* sx
                        const float* topk_w, const void* w1q, const float* s1, const void* w3q, const float* s3,
                        const void* w2q, const float* s2, void* o, void* ws, size_t ws_bytes, void* stream);
 
+/* moe_layer with FP8 experts: gate, top-k and layout on the bf16 activations as in moe_layer; x is
+ * quantised per token into the workspace, GEMM-1 gathers the E4M3 rows, h is quantised per row,
+ * GEMM-2 and Combine as in moe_layer.  Weights and scales as for moe_expert_ffn_fp8.  Same flags,
+ * optional outputs and limits as moe_layer, plus d % 16 == 0 and f % 16 == 0. */
+int moe_layer_fp8(const moe_shape_t* shape, const void* x, const float* w_gate, const float* logit_bias,
+                  int64_t bias_row_stride, const void* w1q, const float* s1, const void* w3q, const float* s3,
+                  const void* w2q, const float* s2, void* y, float* logits, int32_t* topk_idx, float* topk_w,
+                  const moe_layout_t* layout, void* ws, size_t ws_bytes, void* stream);
+
 /* Dispatch without a workspace (the paper has no counterpart; this entry point exists for
  * callers that cannot supply scratch memory).  Some users of this library run where device
  * memory cannot be obtained around the call: plugins that execute inside a host framework's

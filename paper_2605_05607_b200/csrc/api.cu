@@ -14,7 +14,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Regions of the workspace, in order.  Every region starts on a 1 KiB boundary.
 struct WsPlan {
-  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, wsplit, h, hq, sh, o, logits, topk_idx, topk_w;
+  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, wsplit, h, hq, sh, xq, sx, o, logits, topk_idx, topk_w;
   size_t expert_counts, expert_offsets, group_counts, group_offsets, pair_row, row_pair, al, disp_token, row_src;
   size_t total;
   int W;
@@ -46,6 +46,8 @@ WsPlan plan(const moe_shape_t& s) {
   p.h = take(P * (size_t)s.f * 2);
   p.hq = take(P * (size_t)s.f);   // FP8 form: E4M3 copy of h and its row scales
   p.sh = take(P * 4);
+  p.xq = take(T * (size_t)s.d);   // FP8 layer: E4M3 copy of x and its row scales
+  p.sx = take(T * 4);
   // o [P, d] bf16, or the fp32 token accumulators [T, d] of the Combine-in-epilogue form
   p.o = take((P * 2 > T * 4 ? P * 2 : T * 4) * (size_t)s.d);
   p.logits = take(T * E * 4);
@@ -393,11 +395,20 @@ int moe_combine(const moe_shape_t* shape, const void* o, const moe_layout_t* lay
   return MOE_OK;
 }
 
-int moe_layer(const moe_shape_t* shape, const void* x, const float* w_gate, const float* logit_bias,
-              int64_t bias_row_stride, const void* w1, const void* w3, const void* w2, void* y, float* logits,
-              int32_t* topk_idx, float* topk_w, const moe_layout_t* layout, void* ws, size_t ws_bytes, void* stream) {
+// Shared body of moe_layer and moe_layer_fp8.  fp8 == nullptr: bf16 experts, w1 / w3 / w2 are
+// [E, K, N] bf16.  Otherwise they are E4M3 codes [E, N, K] with the scales in *fp8 (sx, hq, sh are
+// filled here from the workspace).
+static int layer_impl(const moe_shape_t* shape, const void* x, const float* w_gate, const float* logit_bias,
+                      int64_t bias_row_stride, const void* w1, const void* w3, const void* w2, const Fp8Args* fp8,
+                      void* y, float* logits, int32_t* topk_idx, float* topk_w, const moe_layout_t* layout, void* ws,
+                      size_t ws_bytes, void* stream) {
   int rc = check_shape(shape);
   if (rc != MOE_OK) return rc;
+  if (fp8 != nullptr) {
+    if (shape->d % 16 != 0 || shape->f % 16 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
+    if (fp8->s1 == nullptr || fp8->s3 == nullptr || fp8->s2 == nullptr) return MOE_ERR_INVALID_ARG;
+    if (!aligned(fp8->s1, 4) || !aligned(fp8->s3, 4) || !aligned(fp8->s2, 4)) return MOE_ERR_MISALIGNED;
+  }
   if (x == nullptr || w_gate == nullptr || w1 == nullptr || w3 == nullptr || w2 == nullptr || y == nullptr)
     return MOE_ERR_INVALID_ARG;
   if (bias_row_stride != 0 && bias_row_stride != shape->E) return MOE_ERR_INVALID_ARG;
@@ -433,6 +444,15 @@ int moe_layer(const moe_shape_t* shape, const void* x, const float* w_gate, cons
   TCMOE_CUDA(launch_layout(s, idx, L, sc, status, st, /*masks_cleared=*/s.T > 0));
   FfnArgs a{};
   a.a_src = x;
+  Fp8Args q{};
+  if (fp8 != nullptr) {   // experts read the E4M3 copy of x
+    q = *fp8;
+    q.sx = at<float>(ws, p.sx);
+    q.hq = at<void>(ws, p.hq);
+    q.sh = at<float>(ws, p.sh);
+    a.a_src = at<void>(ws, p.xq);
+    TCMOE_CUDA(launch_quantize_rows(x, s.T, s.d, at<void>(ws, p.xq), at<float>(ws, p.sx), st));
+  }
   a.gather_idx = L.row_pair;   // token of expert row r = row_pair[r] / k
   a.gather_div = s.k;
   a.w1 = w1;
@@ -450,13 +470,32 @@ int moe_layer(const moe_shape_t* shape, const void* x, const float* w_gate, cons
     // o never materialises: GEMM-2 adds each weighted row into its token's fp32 accumulator
     a.y_acc = at<float>(ws, p.o);
     if (s.T > 0) TCMOE_CUDA(cudaMemsetAsync(a.y_acc, 0, (size_t)s.T * s.d * 4, st));
-    TCMOE_CUDA(launch_expert_ffn(s, a, st));
+    TCMOE_CUDA(fp8 != nullptr ? launch_expert_ffn_fp8(s, a, q, st) : launch_expert_ffn(s, a, st));
     TCMOE_CUDA(launch_round_rows(s, a.y_acc, y, st));
     return MOE_OK;
   }
-  TCMOE_CUDA(launch_expert_ffn(s, a, st));
+  TCMOE_CUDA(fp8 != nullptr ? launch_expert_ffn_fp8(s, a, q, st) : launch_expert_ffn(s, a, st));
   TCMOE_CUDA(launch_combine(s, a.o, L, idx, tw, nullptr, y, st));
   return MOE_OK;
+}
+
+int moe_layer(const moe_shape_t* shape, const void* x, const float* w_gate, const float* logit_bias,
+              int64_t bias_row_stride, const void* w1, const void* w3, const void* w2, void* y, float* logits,
+              int32_t* topk_idx, float* topk_w, const moe_layout_t* layout, void* ws, size_t ws_bytes, void* stream) {
+  return layer_impl(shape, x, w_gate, logit_bias, bias_row_stride, w1, w3, w2, nullptr, y, logits, topk_idx, topk_w,
+                    layout, ws, ws_bytes, stream);
+}
+
+int moe_layer_fp8(const moe_shape_t* shape, const void* x, const float* w_gate, const float* logit_bias,
+                  int64_t bias_row_stride, const void* w1q, const float* s1, const void* w3q, const float* s3,
+                  const void* w2q, const float* s2, void* y, float* logits, int32_t* topk_idx, float* topk_w,
+                  const moe_layout_t* layout, void* ws, size_t ws_bytes, void* stream) {
+  Fp8Args q{};
+  q.s1 = s1;
+  q.s3 = s3;
+  q.s2 = s2;
+  return layer_impl(shape, x, w_gate, logit_bias, bias_row_stride, w1q, w3q, w2q, &q, y, logits, topk_idx, topk_w,
+                    layout, ws, ws_bytes, stream);
 }
 
 int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, const float* w_gate,

@@ -39,7 +39,9 @@ constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int NUM_BARS = 2 * NSTAGE + 4;
 constexpr int STAGE_OUT_WARP = 32 * 144;     // epilogue transpose buffer of one warp: 32 rows x (128 + 16) bytes
 constexpr int TABLE_BYTES = (2 * (MAX_E + 1) * 4 + 15) & ~15;
-constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + TABLE_BYTES + 4 * STAGE_OUT_WARP;
+constexpr int COLSCALE_WARP = UMMA_N * 4;     // FP8: one warp's copy of the tile's 128 + 128 output-column scales
+constexpr int SMEM_BYTES =
+    1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + TABLE_BYTES + 4 * STAGE_OUT_WARP + 4 * COLSCALE_WARP;
 constexpr int THREADS = 320;
 constexpr int GATHER_THREADS = 128;
 constexpr int BN_OUT = 128;
@@ -61,6 +63,7 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
   int* tp_s = reinterpret_cast<int*>(tmem_slot + 16);
   int* eoff_s = tp_s + (MAX_E + 1);
   const uint32_t stage_base = ptx::smem_u32(tp_s) + TABLE_BYTES;   // 16-byte aligned
+  float* colscale_base = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(tp_s) + TABLE_BYTES + 4 * STAGE_OUT_WARP);
 
   const uint32_t smem_base = ptx::smem_u32(smem);
   const uint32_t bar_base = ptx::smem_u32(bars);
@@ -129,7 +132,8 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
       const uint32_t stage = stage_base + (uint32_t)(warp * STAGE_OUT_WARP);
       const int srow = lane >> 3, piece = lane & 7;
       float sa = 1.f;   // FP8: scale of this thread's row (the gather source row)
-      const float *s1 = nullptr, *s3 = nullptr;
+      float* s1 = colscale_base + warp * UMMA_N;   // this warp's copy of the W1 / W3 column scales (0 beyond N)
+      float* s3 = s1 + 128;
       if (FP8) {
         const int lrow = warp * 32 + lane;
         if (lrow < t.rows) {
@@ -137,8 +141,15 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
           if (p.gather_div > 1) idx /= p.gather_div;
           sa = __ldg(p.a_scale + idx);
         }
-        s1 = p.b_scale + (size_t)t.e * p.N + t.n0;
-        s3 = p.b_scale2 + (size_t)t.e * p.N + t.n0;
+        const size_t g = (size_t)t.e * p.N + t.n0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int n = lane + 32 * i;
+          const bool in = t.n0 + n < p.N;
+          s1[n] = in ? (__ldg(p.b_scale + g + n)) : 0.f;
+          s3[n] = in ? (__ldg(p.b_scale2 + g + n)) : 0.f;
+        }
+        __syncwarp();
       }
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
@@ -156,11 +167,10 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
             float g0 = __uint_as_float(a3[j]), g1 = __uint_as_float(a3[j + 1]);
             if (FP8) {
               const int n = c * 32 + j;
-              const bool in0 = t.n0 + n < p.N, in1 = t.n0 + n + 1 < p.N;
-              u0 *= sa * (in0 ? __ldg(s1 + n) : 0.f);
-              g0 *= sa * (in0 ? __ldg(s3 + n) : 0.f);
-              u1 *= sa * (in1 ? __ldg(s1 + n + 1) : 0.f);
-              g1 *= sa * (in1 ? __ldg(s3 + n + 1) : 0.f);
+              u0 *= sa * s1[n];
+              g0 *= sa * s3[n];
+              u1 *= sa * s1[n + 1];
+              g1 *= sa * s3[n + 1];
             }
             q[i] = pack2(silu_mul(u0, g0), silu_mul(u1, g1));
           }

@@ -31,7 +31,9 @@ constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int NUM_BARS = 2 * NSTAGE + 4;
 constexpr int STAGE_OUT_WARP = 32 * 144;          // epilogue transpose buffer of one warp: 32 rows x (128 + 16) bytes
 constexpr int TABLE_BYTES = (2 * (MAX_E + 1) * 4 + 15) & ~15;
-constexpr int SMEM_BYTES = 1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + TABLE_BYTES + 4 * STAGE_OUT_WARP;
+constexpr int COLSCALE_WARP = UMMA_N * 4;          // FP8: one warp's copy of the tile's 256 output-column scales
+constexpr int SMEM_BYTES =
+    1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + TABLE_BYTES + 4 * STAGE_OUT_WARP + 4 * COLSCALE_WARP;
 constexpr int THREADS = 192;
 constexpr int BN_OUT = 256;
 constexpr uint32_t IDESC = idesc_bf16(2 * BM);
@@ -56,6 +58,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
   int* tp_s = reinterpret_cast<int*>(tmem_slot + 16);
   int* eoff_s = tp_s + (MAX_E + 1);
   const uint32_t stage_base = ptx::smem_u32(tp_s) + TABLE_BYTES;   // 16-byte aligned
+  float* colscale_base = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(tp_s) + TABLE_BYTES + 4 * STAGE_OUT_WARP);
 
   const uint32_t smem_base = ptx::smem_u32(smem);
   const uint32_t bar_base = ptx::smem_u32(bars);
@@ -131,7 +134,18 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
         if (FP8) wr *= __ldg(p.a_scale + grow);   // row scale of h joins the gate weight
         if (RED) yrow = p.y_acc + (size_t)(pair / p.y_div) * (size_t)p.N + t.n0;
       }
-      const float* sb_col = FP8 ? p.b_scale + (size_t)t.e * p.N + t.n0 : nullptr;
+      // FP8: the tile's output-column scales, one copy per warp (0 beyond N), staged while the
+      // main loop of this tile may still be running
+      float* sb_col = colscale_base + warp * UMMA_N;
+      if (FP8) {
+        const float* g = p.b_scale + (size_t)t.e * p.N + t.n0;
+#pragma unroll
+        for (int i = 0; i < UMMA_N / 32; ++i) {
+          const int n = lane + 32 * i;
+          sb_col[n] = (t.n0 + n < p.N) ? __ldg(g + n) : 0.f;
+        }
+        __syncwarp();
+      }
       if (RED) {
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
@@ -142,7 +156,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               const int n = c * 32 + j;
-              acc[j] = __float_as_uint(__uint_as_float(acc[j]) * (t.n0 + n < p.N ? __ldg(sb_col + n) : 0.f));
+              acc[j] = __float_as_uint(__uint_as_float(acc[j]) * sb_col[n]);
             }
           }
           if (valid) {
@@ -176,8 +190,8 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               const int n = cc * 64 + j;
-              acc0[j] = __float_as_uint(__uint_as_float(acc0[j]) * (t.n0 + n < p.N ? __ldg(sb_col + n) : 0.f));
-              acc1[j] = __float_as_uint(__uint_as_float(acc1[j]) * (t.n0 + n + 32 < p.N ? __ldg(sb_col + n + 32) : 0.f));
+              acc0[j] = __float_as_uint(__uint_as_float(acc0[j]) * sb_col[n]);
+              acc1[j] = __float_as_uint(__uint_as_float(acc1[j]) * sb_col[n + 32]);
             }
           }
 #pragma unroll

@@ -93,3 +93,39 @@ def test_fp8_shape_limits():
     with pytest.raises(B.MoEError) as ei:
         B.moe_expert_ffn_fp8(run.shape, z8, zf, run.lay, zf, z8, zf, z8, zf, z8, zf, run.o, run.ws)
     assert ei.value.code == B.MOE_ERR_UNSUPPORTED_SHAPE
+
+
+def _quantized_weights(t, cfg):
+    E, d, f = cfg.E, cfg.d, cfg.f
+    wq, sc = {}, {}
+    for name, (K, N) in (("w1", (d, f)), ("w3", (d, f)), ("w2", (f, d))):
+        wq[name] = torch.zeros(E, N, K, dtype=torch.uint8, device="cuda")
+        sc[name] = torch.zeros(E, N, dtype=torch.float32, device="cuda")
+        B.moe_quantize_weights(t[name], wq[name], sc[name])
+    return wq, sc
+
+
+@pytest.mark.parametrize("cfg", FP8_CASES, ids=lambda c: c.name)
+@pytest.mark.parametrize("flags", [0, B.MOE_FLAG_COMBINE_IN_EPILOGUE], ids=["combine-kernel", "combine-in-epilogue"])
+def test_layer_fp8_matches_its_oracle(cfg, flags):
+    run = H.Run(cfg, flags)
+    t = run.t
+    wq, sc = _quantized_weights(t, cfg)
+    lay_dev = B.alloc_layout(run.shape)
+    for _ in range(2):
+        run.y.fill_(3.0)
+        B.moe_layer_fp8(run.shape, t["x"], t["w_gate"], t["bias"], wq["w1"], sc["w1"], wq["w3"], sc["w3"], wq["w2"],
+                        sc["w2"], run.y, run.ws, logits=run.logits, topk_idx=run.idx, topk_w=run.w, layout=lay_dev)
+    torch.cuda.synchronize()
+    assert run.status()[0] == 0
+    run.lay = lay_dev
+    idx_ref, _ = H.check_route(run)          # routing runs on the bf16 activations, as in moe_layer
+    lay = H.check_layout(run, idx_ref)
+    # per-token quantisation commutes with the dispatch copy: quantise x, then take the dispatched rows
+    xq, sx = F.quantize_rows(O.bf16_to_f64(H.bf16_host(t["x"])))
+    dt = lay["disp_token"].astype(np.int64)
+    ref_w = {n: F.quantize_weights(O.bf16_to_f64(H.bf16_host(t[n]))) for n in ("w1", "w3", "w2")}
+    o_ref = F.expert_ffn_fp8(xq[dt], sx[dt], lay, run.host_w(), *ref_w["w1"], *ref_w["w3"], *ref_w["w2"])
+    _, _, y_ref = O.combine(o_ref, lay, idx_ref, None, cfg.E, cfg.G)
+    y_gpu = O.bf16_to_f64(H.bf16_host(run.y)[: cfg.T])
+    H.assert_close_out(y_gpu, y_ref, "fp8 layer y")
