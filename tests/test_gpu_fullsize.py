@@ -80,3 +80,75 @@ def test_fullsize_layer(name):
                              k, cfg.score_fn, tokens=few)
     y_few = O.bf16_to_f64(H.bf16_host(run.y[torch.from_numpy(few).cuda()]))
     H.assert_close_out(y_few, y_def, f"{name} layer y")
+
+
+class QuantSlabs:
+    """Per-expert FP8 weights computed by the oracle from the bf16 slab of that expert only."""
+
+    def __init__(self, w, which):
+        from oracle import fp8_oracle as F
+        self.w, self.which, self.F, self.cache = w, which, F, {}
+        self.shape = (w.shape[0], w.shape[2], w.shape[1])          # [E, N, K]
+
+    def __getitem__(self, e):
+        e = int(e)
+        if e not in self.cache:
+            q, s = self.F.quantize_weights(O.bf16_to_f64(synth.bf16_bits(self.w[e]))[None])
+            self.cache[e] = (q[0], s[0])
+        return self.cache[e][self.which]
+
+
+@pytest.mark.parametrize("name", ["C4", "S32"])
+def test_fullsize_layer_fp8(name):
+    """moe_layer_fp8 at full size: routing and layout in full, quantised operands bit for bit on
+    sampled experts, expert outputs on sampled rows and the layer output on sampled tokens."""
+    from oracle import fp8_oracle as F
+    cfg = synth.ALL_CONFIGS[name]
+    run = H.Run(cfg)
+    t = run.t
+    E, d, f, P, T, k = cfg.E, cfg.d, cfg.f, cfg.P, cfg.T, cfg.k
+    wq, sc = {}, {}
+    for nm, (K, N) in (("w1", (d, f)), ("w3", (d, f)), ("w2", (f, d))):
+        wq[nm] = torch.zeros(E, N, K, dtype=torch.uint8, device="cuda")
+        sc[nm] = torch.zeros(E, N, dtype=torch.float32, device="cuda")
+        B.moe_quantize_weights(t[nm], wq[nm], sc[nm])
+    lay_dev = B.alloc_layout(run.shape)
+    B.moe_layer_fp8(run.shape, t["x"], t["w_gate"], t["bias"], wq["w1"], sc["w1"], wq["w3"], sc["w3"], wq["w2"],
+                    sc["w2"], run.y, run.ws, logits=run.logits, topk_idx=run.idx, topk_w=run.w, layout=lay_dev)
+    torch.cuda.synchronize()
+    st = run.status()
+    assert st[0] == 0 and st[4] == 0, f"device status {st}"
+    run.lay = lay_dev
+    idx_ref, _ = H.check_route(run)
+    lay = H.check_layout(run, idx_ref)
+    counts = lay["expert_counts"]
+    live = np.nonzero(counts)[0]
+    rng = np.random.default_rng(2)
+    picks = sorted({int(live[np.argmax(counts[live])]), int(live[np.argmin(counts[live])]), int(rng.choice(live))})
+    slabs = {nm: (QuantSlabs(t[nm], 0), QuantSlabs(t[nm], 1)) for nm in ("w1", "w3", "w2")}
+    for e in picks:      # the GPU's quantised weights of the sampled experts, bit for bit
+        for nm in ("w1", "w3", "w2"):
+            assert np.array_equal(wq[nm][e].cpu().numpy(), slabs[nm][0][e]), (nm, e)
+            assert np.array_equal(sc[nm][e].cpu().numpy(), slabs[nm][1][e]), (nm, e)
+    rows = []
+    for e in picks:
+        lo, hi = int(lay["expert_offsets"][e]), int(lay["expert_offsets"][e + 1])
+        rows.append(np.unique(np.concatenate([np.arange(lo, min(lo + 6, hi)), np.arange(max(hi - 6, lo), hi),
+                                              rng.integers(lo, hi, size=6)])))
+    rows = np.unique(np.concatenate(rows))
+    xq, sx = F.quantize_rows(O.bf16_to_f64(H.bf16_host(t["x"])))
+    dt = lay["disp_token"].astype(np.int64)
+    o_ref = F.expert_ffn_fp8(xq[dt], sx[dt], lay, run.host_w(), slabs["w1"][0], slabs["w1"][1], slabs["w3"][0],
+                             slabs["w3"][1], slabs["w2"][0], slabs["w2"][1], rows=rows)
+    off = B.moe_workspace_layout(run.shape)
+    o_dev = run.ws[off["o"]: off["o"] + P * d * 2].view(torch.bfloat16).reshape(P, d)
+    o_gpu = O.bf16_to_f64(H.bf16_host(o_dev[torch.from_numpy(rows).cuda()]))
+    H.assert_close_out(o_gpu, o_ref, f"{name} fp8 expert rows")
+    # combine on sampled tokens from the GPU's own o
+    toks = synth.sample_tokens(cfg, 64)
+    need = np.unique(lay["pair_row"].reshape(T, k)[toks].reshape(-1))
+    o_need = O.bf16_to_f64(H.bf16_host(o_dev[torch.from_numpy(need).cuda()]))
+    _, _, y_ref = O.combine(o_need, lay, idx_ref, None, E, cfg.G, tokens=toks, o_rows=need)
+    y_gpu = O.bf16_to_f64(H.bf16_host(run.y[torch.from_numpy(toks).cuda()]))
+    tol = 2.0 ** -8 * np.abs(y_ref) + 2.0 ** -22 * np.abs(y_ref).max() + 1e-30
+    assert np.all(np.abs(y_gpu - y_ref) <= tol), f"{name} fp8 combine"
