@@ -266,6 +266,37 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
         B.moe_profile_enable(0)
         out["layer_fused"][kn + "_in_layer_ms"] = ms / max(n, 1)
     out["combine"]["in_layer_gbs"] = comb_bytes / out["layer_fused"]["combine_in_layer_ms"] / 1e6
+    # FP8 experts (E4M3, per-token and per-output-column scales): the same layer through moe_layer_fp8
+    if d % 16 == 0 and f % 16 == 0:
+        wq, sc = {}, {}
+        for nm, (K, N) in (("w1", (d, f)), ("w3", (d, f)), ("w2", (f, d))):
+            wq[nm] = torch.zeros(E, N, K, dtype=torch.uint8, device=dev)
+            sc[nm] = torch.zeros(E, N, dtype=torch.float32, device=dev)
+            B.moe_quantize_weights(t[nm], wq[nm], sc[nm])
+
+        def layer_fp8():
+            B.moe_layer_fp8(shape, t["x"], t["w_gate"], t["bias"], wq["w1"], sc["w1"], wq["w3"], sc["w3"], wq["w2"],
+                            sc["w2"], y, ws)
+
+        layer_fp8()
+        times = []
+        for _ in range(reps):
+            torch.cuda.synchronize()
+            time.sleep(0.2)
+            times.append(timed(layer_fp8))
+        fp8 = {"ms": float(np.median(times)), "tokens_per_s": T / float(np.median(times)) * 1e3}
+        for kn in ("gemm1", "gemm2"):
+            B.moe_profile_enable(B.KERNEL_IDS[kn])
+            for _ in range(reps):
+                layer_fp8()
+            ms, n = B.moe_profile_read()
+            B.moe_profile_enable(0)
+            fp8[kn + "_in_layer_ms"] = ms / max(n, 1)
+        fp8["gemm1_tflops"] = 4.0 * P * d * f / fp8["gemm1_in_layer_ms"] / 1e9
+        fp8["gemm2_tflops"] = 2.0 * P * d * f / fp8["gemm2_in_layer_ms"] / 1e9
+        fp8["note"] = "E4M3 experts, bf16 gate / combine; includes per-token quantisation of x and per-row quantisation of h"
+        out["layer_fp8"] = fp8
+        del wq, sc
     out["inputs"] = {"seed": cfg.seed, "sub_streams": "seed*1000 + tensor id",
                      "checksums": {n: synth.tensor_checksum(t[n]) for n in ("x", "w_gate", "bias", "w1", "w3", "w2")}}
     out["summary"] = {"unfused_sum_ms": unfused, "unfused_back_to_back_ms": float(np.median(seq_ms)),
