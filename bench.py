@@ -337,6 +337,9 @@ def main():
     ap.add_argument("--ref-sample", type=int, default=0,
                     help="tokens per step of the reference arm (0: sized from a one-token calibration)")
     ap.add_argument("--cpu-sample", type=int, default=64, help="tokens of the cpu_baseline leg (0: skip)")
+    ap.add_argument("--experts", default="bf16", choices=["bf16", "fp8"],
+                    help="bf16 (the benchmark's precision, default) or fp8: E4M3 experts through moe_layer_fp8 "
+                         "(per-token / per-output-column scales; gate and combine stay bf16 / fp32)")
     ap.add_argument("--lean", action="store_true",
                     help="timed region only: no e2e / stage / cpu_baseline legs (for profiler captures)")
     ap.add_argument("--stages-only", action="store_true",
@@ -383,8 +386,23 @@ def main():
     ws = B.alloc_workspace(shape)
     y = torch.zeros(cfg.T, cfg.d, dtype=torch.bfloat16, device="cuda")
 
+    fp8 = args.experts == "fp8"
+    if fp8:   # static weights are quantised once, outside the timed region; x is quantised inside every step
+        wq, sc = {}, {}
+        for nm, (K, N) in (("w1", (cfg.d, cfg.f)), ("w3", (cfg.d, cfg.f)), ("w2", (cfg.f, cfg.d))):
+            wq[nm] = torch.zeros(cfg.E, N, K, dtype=torch.uint8, device="cuda")
+            sc[nm] = torch.zeros(cfg.E, N, dtype=torch.float32, device="cuda")
+            B.moe_quantize_weights(t[nm], wq[nm], sc[nm])
+
+    def layer(x, y_out, work, stream=None):
+        if fp8:
+            B.moe_layer_fp8(shape, x, t["w_gate"], t["bias"], wq["w1"], sc["w1"], wq["w3"], sc["w3"], wq["w2"],
+                            sc["w2"], y_out, work, stream=stream)
+        else:
+            B.moe_layer(shape, x, t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y_out, work, stream=stream)
+
     def step():
-        B.moe_layer(shape, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws)
+        layer(t["x"], y, ws)
 
     sampler = None
     if rank == 0:
@@ -432,13 +450,18 @@ def main():
 
         def step_host(i):
             ln = lanes[i & 1]
-            B.moe_layer_host(shape, x_host, ln["x_dev"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"],
-                             ln["y_dev"], ln["y_host"], ln["ws"], stream=ln["stream"])
+            if fp8:   # no host-buffer entry point for the FP8 layer: the same copies, issued from here
+                with torch.cuda.stream(ln["stream"]):
+                    ln["x_dev"].copy_(x_host, non_blocking=True)
+                    layer(ln["x_dev"], ln["y_dev"], ln["ws"], stream=ln["stream"])
+                    ln["y_host"].copy_(ln["y_dev"], non_blocking=True)
+            else:
+                B.moe_layer_host(shape, x_host, ln["x_dev"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"],
+                                 ln["y_dev"], ln["y_host"], ln["ws"], stream=ln["stream"])
 
         def step_dev(i):   # same two-stream schedule without the copies, for comparison
             ln = lanes[i & 1]
-            B.moe_layer(shape, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], ln["y_dev"], ln["ws"],
-                        stream=ln["stream"])
+            layer(t["x"], ln["y_dev"], ln["ws"], stream=ln["stream"])
 
         main = torch.cuda.current_stream()
 
@@ -490,29 +513,34 @@ def main():
     flops_g1 = 4.0 * cfg.P * cfg.d * cfg.f                      # GEMM-1: x W1 and x W3
     g1_avg_s = (g1_ms / max(g1_launches, 1)) * 1e-3
     achieved = flops_g1 / g1_avg_s / 1e12 if g1_launches else None
-    peak = pk["bf16_tflops_sustained"]
+    peak = pk["bf16_tflops_sustained"] * (2.0 if fp8 else 1.0)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic", "config": workload_config(cfg, world),
+        "dtype": "fp8" if fp8 else "bf16", "data": "synthetic", "config": workload_config(cfg, world),
         "clocks": clocks,
         "e2e": None if e2e_ms is None else
                {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.T * cfg.d * 2,
                 "d2h_bytes_per_step": cfg.T * cfg.d * 2,
                 "pipeline": "moe_layer_host on 2 alternating streams (double-buffered staging and workspace)"},
         "value_two_streams": None if two_stream_ms is None else tokens / (two_stream_ms * 1e-3),
-        "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "gpu_launches": (KERNELS_PER_STEP + (2 if fp8 else 0)) * args.steps,   # FP8: + quantisation of x and of h
         "roofline": {"kernel": "ffn_gemm1_kernel (GEMM-1 + SwiGLU, tcgen05)", "bound": "tensor",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": (achieved / peak) if achieved else None,
-                     "peak_source": f"{pk['source']} bf16 sustained (kernel timed inside a long step)",
+                     "peak_source": f"{pk['source']} bf16 sustained (kernel timed inside a long step)" +
+                                    (" x 2 (nominal fp8 : bf16 ratio; no measured fp8 peak)" if fp8 else ""),
                      "flops_per_launch": flops_g1, "avg_launch_ms": g1_avg_s * 1e3, "launches": g1_launches,
-                     "traffic": GEMM1_DRAM_TRAFFIC.get(cfg.name)},
+                     "traffic": None if fp8 else GEMM1_DRAM_TRAFFIC.get(cfg.name)},
         "ffn_tflops_layer": 6.0 * cfg.P * cfg.d * cfg.f * args.steps / (elapsed_ms * 1e-3) / 1e12,
         "paper_context": "the paper reports only relative figures: up to 1.79x end-to-end training speedup over COMET "
                          "(geomean 1.59x) on a SIMULATED 32-GPU GH200 NVL32 (BookSim2 + Accel-Sim, H200-configured "
                          "GPUs, NVLink 4, FP8 GEMMs); no tokens/s, GB/s or TFLOP/s for this path, hence vs_baseline null",
     }
+    if fp8:
+        line["experts"] = ("E4M3 weights and activations, one fp32 scale per token / per (expert, output column), "
+                           "fp32 accumulation; a reduced-precision variant, not the benchmark's bf16 configuration")
+        del wq, sc
     if world == 1 and not args.lean:
         line["stages"] = stage_breakdown(cfg, t)
     if world == 1 and args.report and not args.lean:
