@@ -2,18 +2,23 @@
 // (GEMM-1 + SwiGLU in ffn_gemm1.cu, GEMM-2 + gate weight in ffn_gemm2.cu).
 #include "ffn_common.cuh"
 
+#include <atomic>
+
 namespace tcmoe {
 
 namespace {
 
 ffn::EncodeTiledFn encode_fn() {
-  static ffn::EncodeTiledFn fn = nullptr;
+  static std::atomic<ffn::EncodeTiledFn> cached{nullptr};   // looked up once; a second lookup gives the same address
+  ffn::EncodeTiledFn fn = cached.load(std::memory_order_acquire);
   if (fn == nullptr) {
     void* sym = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
+        q == cudaDriverEntryPointSuccess) {
       fn = reinterpret_cast<ffn::EncodeTiledFn>(sym);
+      cached.store(fn, std::memory_order_release);
+    }
   }
   return fn;
 }
@@ -82,15 +87,17 @@ int current_device() {
 }
 
 int sm_count() {
-  static int n[MAX_DEVICES] = {};
+  static std::atomic<int> cached[MAX_DEVICES];
   const int dev = current_device();
-  if (n[dev] == 0) {
-    if (cudaDeviceGetAttribute(&n[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n[dev] <= 0) {
+  int n = cached[dev].load(std::memory_order_relaxed);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
       (void)cudaGetLastError();
-      n[dev] = 148;
+      n = 148;
     }
+    cached[dev].store(n, std::memory_order_relaxed);
   }
-  return n[dev];
+  return n;
 }
 
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st) {

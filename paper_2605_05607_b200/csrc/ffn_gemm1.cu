@@ -28,6 +28,8 @@
 // depth, and TMA tile::gather4 sustains only one 4-row instruction per ~40 ns.
 #include "ffn_common.cuh"
 
+#include <atomic>
+
 namespace tcmoe {
 namespace ffn {
 namespace {
@@ -321,14 +323,15 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
 
 cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, bool fp8,
                          cudaStream_t st) {
-  static bool attr_set[MAX_DEVICES] = {};   // the attribute is per device
+  // per device; several host threads may get here at once: setting the attribute twice is harmless
+  static std::atomic<bool> attr_set[MAX_DEVICES];
   const int dev = current_device();
-  if (!attr_set[dev]) {
+  if (!attr_set[dev].load(std::memory_order_acquire)) {
     cudaError_t e = cudaFuncSetAttribute(ffn_gemm1_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(ffn_gemm1_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set[dev] = true;
+    attr_set[dev].store(true, std::memory_order_release);
   }
   ProfileScope prof(KID_GEMM1, st);
   if (fp8) return launch_pdl(ffn_gemm1_kernel<true>, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);

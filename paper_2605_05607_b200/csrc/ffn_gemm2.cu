@@ -20,6 +20,8 @@
 // peer has stopped touching its shared memory and TMEM (cluster barrier at the end).
 #include "ffn_common.cuh"
 
+#include <atomic>
+
 namespace tcmoe {
 namespace ffn {
 namespace {
@@ -312,8 +314,9 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
 
 // Persistent grid: two CTAs per resident cluster, at most one CTA per SM.
 int pair_grid() {
-  static int grid_of[MAX_DEVICES] = {};
-  int& g = grid_of[current_device()];
+  static std::atomic<int> grid_of[MAX_DEVICES];   // 0 = not computed yet; recomputing gives the same value
+  std::atomic<int>& cached = grid_of[current_device()];
+  int g = cached.load(std::memory_order_relaxed);
   if (g == 0) {
     int clusters = 0;
     cudaLaunchConfig_t cfg = {};
@@ -332,6 +335,7 @@ int pair_grid() {
       clusters = sm_count() / 2;
     }
     g = 2 * min(clusters, sm_count() / 2);
+    cached.store(g, std::memory_order_relaxed);
   }
   return g;
 }
@@ -340,16 +344,17 @@ int pair_grid() {
 
 cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, bool fp8,
                          cudaStream_t st) {
-  static bool attr_set[MAX_DEVICES] = {};   // the attribute is per device
+  // per device; several host threads may get here at once: setting the attribute twice is harmless
+  static std::atomic<bool> attr_set[MAX_DEVICES];
   const int dev = current_device();
-  if (!attr_set[dev]) {
+  if (!attr_set[dev].load(std::memory_order_acquire)) {
     const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
     cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false>, attr, SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, false>, attr, SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, true>, attr, SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, true>, attr, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set[dev] = true;
+    attr_set[dev].store(true, std::memory_order_release);
   }
   ProfileScope prof(KID_GEMM2, st);
   const bool red = p.y_acc != nullptr;

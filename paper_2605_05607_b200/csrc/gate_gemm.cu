@@ -17,6 +17,8 @@
 //    4 stages (the accumulators of 3 x 256 columns would not fit the 512 TMEM columns).
 #include "ffn_common.cuh"
 
+#include <atomic>
+
 namespace tcmoe {
 namespace {
 
@@ -218,13 +220,16 @@ gate_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
 }
 
 EncodeTiledFn encoder() {
-  static EncodeTiledFn fn = nullptr;
+  static std::atomic<EncodeTiledFn> cached{nullptr};   // looked up once; a second lookup gives the same address
+  EncodeTiledFn fn = cached.load(std::memory_order_acquire);
   if (fn == nullptr) {
     void* sym = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
+        q == cudaDriverEntryPointSuccess) {
       fn = reinterpret_cast<EncodeTiledFn>(sym);
+      cached.store(fn, std::memory_order_release);
+    }
   }
   return fn;
 }
@@ -236,12 +241,13 @@ size_t gate_split_bytes(int d, int E) { return (size_t)3 * d * ((E + 63) & ~63) 
 cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gate, float* logits, void* wsplit,
                                int32_t* status, cudaStream_t st) {
   if (s.T == 0) return cudaSuccess;
-  static bool attr_set[MAX_DEVICES] = {};   // the attribute is per device
+  // per device; several host threads may get here at once: setting the attribute twice is harmless
+  static std::atomic<bool> attr_set[MAX_DEVICES];
   const int dev = current_device();
-  if (!attr_set[dev]) {
+  if (!attr_set[dev].load(std::memory_order_acquire)) {
     cudaError_t e = cudaFuncSetAttribute(gate_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_set[dev] = true;
+    attr_set[dev].store(true, std::memory_order_release);
   }
   const int Epad = (s.E + 63) & ~63;
   EncodeTiledFn fn = encoder();
