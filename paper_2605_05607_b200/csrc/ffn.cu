@@ -2,6 +2,8 @@
 // (GEMM-1 + SwiGLU in ffn_gemm1.cu, GEMM-2 + gate weight in ffn_gemm2.cu).
 #include "ffn_common.cuh"
 
+#include <cstdlib>
+
 #include <atomic>
 
 namespace tcmoe {
@@ -100,6 +102,16 @@ int sm_count() {
   return n;
 }
 
+// Experts holding few rows on average: 256-row CTA-pair tiles would be mostly padding (a Zipf-routed
+// 128-expert layer has most experts below 128 rows), so GEMM-2 takes 128-row single-CTA tiles.  Decided from the
+// shape alone (the routing-dependent counts never visit the host); TCMOE_GEMM2=pair|single overrides for experiments.
+static bool small_experts(const Shape& s) {
+  const char* env = getenv("TCMOE_GEMM2");
+  if (env != nullptr && env[0] == 'p') return false;
+  if (env != nullptr && env[0] == 's') return true;
+  return (long long)s.T * s.k < 512ll * s.E;
+}
+
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st) {
   if (s.T == 0) return cudaSuccess;
   const int P = s.T * s.k;
@@ -139,6 +151,12 @@ cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st)
   g2.status = a.status;
   g2.y_acc = a.y_acc;
   g2.y_div = s.k;
+  if (small_experts(s) && a.y_acc == nullptr) {
+    g2.a_src = a.h;
+    g2.a_ld = s.f;
+    g2.tile_prefix = a.mt_prefix;
+    return ffn::launch_gemm2_single(g2, m_w2, false, st);
+  }
   return ffn::launch_gemm2(g2, m_w2, m_h, false, st);
 }
 
@@ -188,6 +206,12 @@ cudaError_t launch_expert_ffn_fp8(const Shape& s, const FfnArgs& a, const Fp8Arg
   g2.y_div = s.k;
   g2.a_scale = q.sh;
   g2.b_scale = q.s2;
+  if (small_experts(s) && a.y_acc == nullptr) {
+    g2.a_src = q.hq;
+    g2.a_ld = s.f;
+    g2.tile_prefix = a.mt_prefix;
+    return ffn::launch_gemm2_single(g2, m_w2, true, st);
+  }
   return ffn::launch_gemm2(g2, m_w2, m_h, true, st);
 }
 

@@ -113,6 +113,8 @@ cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUt
                          cudaStream_t st);
 cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, bool fp8,
                          cudaStream_t st);
+// GEMM-2 on 128-row single-CTA tiles (small experts): p.a_src / p.a_ld = h rows, no Combine-in-epilogue form
+cudaError_t launch_gemm2_single(const GemmParams& p, const CUtensorMap& m_w2, bool fp8, cudaStream_t st);
 
 }  // namespace ffn
 }  // namespace tcmoe

@@ -53,7 +53,13 @@ constexpr uint32_t IDESC_F8 = idesc_e4m3(BM);
 // FP8 = true: A rows and weights are E4M3 codes, a stage holds 128 elements of K (the same 128
 // bytes per row), W1 / W3 come K-major from [E, N, K] as two 128-row boxes, and the epilogue applies
 // a_scale[source row] * b_scale[e, n] before the SwiGLU; h is written as bf16 either way.
-template <bool FP8>
+//
+// PLAIN = true turns the kernel into a single-CTA form of GEMM-2 (Sec. II-A "GEMM-2", gate weight in the
+// epilogue, Sec. III-C): the "gather" reads the rows of h in place (gather_idx = NULL), both halves of
+// the 256-column B tile come from the one weight map (map_w1), the epilogue writes
+// o[r, n] = w_r * acc[r, n] for 256 columns.  Used instead of the CTA-pair kernel when experts are small
+// (128-row tiles pad far less than 256-row pair tiles when most experts hold fewer than 128 rows).
+template <bool FP8, bool PLAIN>
 __global__ void __launch_bounds__(THREADS, 1)
 ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w3,
                  const GemmParams p) {
@@ -112,11 +118,11 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
   const volatile int* global_abort = p.status + ST_ABORT;
 
   auto timeout = [&](int detail) {
-    report_error(p.status, DEV_TIMEOUT, KID_GEMM1, detail, blockIdx.x);
+    report_error(p.status, DEV_TIMEOUT, PLAIN ? KID_GEMM2 : KID_GEMM1, detail, blockIdx.x);
     p.status[ST_ABORT] = 1;
     *abort_flag = 1;
   };
-  auto tile_of = [&](int w) { return decode_tile(w, tp_s, eoff_s, p.E, p.n_tiles, BN_OUT, BM, 0); };
+  auto tile_of = [&](int w) { return decode_tile(w, tp_s, eoff_s, p.E, p.n_tiles, PLAIN ? 2 * BN_OUT : BN_OUT, BM, 0); };
 
   if (warp < 4) {
     // ================================ epilogue ================================
@@ -133,6 +139,69 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
       // stores whole 128-byte row segments, 8 lanes per row, 4 rows per instruction.
       const uint32_t stage = stage_base + (uint32_t)(warp * STAGE_OUT_WARP);
       const int srow = lane >> 3, piece = lane & 7;
+      if (PLAIN) {
+        // ---- GEMM-2 form: o = (gate weight x row scale) * acc * column scale, 256 columns
+        const int lrow = warp * 32 + lane;
+        float wr = 1.f;
+        if (lrow < t.rows) {
+          const size_t grow = (size_t)t.row0 + lrow;
+          if (p.topk_w != nullptr) wr = __ldg(p.topk_w + __ldg(p.row_pair + grow));
+          if (FP8) wr *= __ldg(p.a_scale + grow);
+        }
+        float* sb_col = colscale_base + warp * UMMA_N;
+        if (FP8) {
+          const float* g = p.b_scale + (size_t)t.e * p.N + t.n0;
+#pragma unroll
+          for (int i = 0; i < UMMA_N / 32; ++i) {
+            const int n = lane + 32 * i;
+            sb_col[n] = (t.n0 + n < p.N) ? __ldg(g + n) : 0.f;
+          }
+          __syncwarp();
+        }
+#pragma unroll 1
+        for (int cc = 0; cc < 4; ++cc) {
+          uint32_t acc0[32], acc1[32];
+          ptx::tmem_ld32(taddr + cc * 64, acc0);
+          ptx::tmem_ld32(taddr + cc * 64 + 32, acc1);
+          ptx::tmem_ld_wait_on(acc0);
+          ptx::tmem_ld_wait_on(acc1);
+          if (FP8) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int n = cc * 64 + j;
+              acc0[j] = __float_as_uint(__uint_as_float(acc0[j]) * sb_col[n]);
+              acc1[j] = __float_as_uint(__uint_as_float(acc1[j]) * sb_col[n + 32]);
+            }
+          }
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            ptx::st_shared_v4(stage + lane * 144 + v * 16,
+                              pack2(wr * __uint_as_float(acc0[v * 8]), wr * __uint_as_float(acc0[v * 8 + 1])),
+                              pack2(wr * __uint_as_float(acc0[v * 8 + 2]), wr * __uint_as_float(acc0[v * 8 + 3])),
+                              pack2(wr * __uint_as_float(acc0[v * 8 + 4]), wr * __uint_as_float(acc0[v * 8 + 5])),
+                              pack2(wr * __uint_as_float(acc0[v * 8 + 6]), wr * __uint_as_float(acc0[v * 8 + 7])));
+            ptx::st_shared_v4(stage + lane * 144 + 64 + v * 16,
+                              pack2(wr * __uint_as_float(acc1[v * 8]), wr * __uint_as_float(acc1[v * 8 + 1])),
+                              pack2(wr * __uint_as_float(acc1[v * 8 + 2]), wr * __uint_as_float(acc1[v * 8 + 3])),
+                              pack2(wr * __uint_as_float(acc1[v * 8 + 4]), wr * __uint_as_float(acc1[v * 8 + 5])),
+                              pack2(wr * __uint_as_float(acc1[v * 8 + 6]), wr * __uint_as_float(acc1[v * 8 + 7])));
+          }
+          __syncwarp();
+          const int col = t.n0 + cc * 64 + piece * 8;
+          if (col < p.N) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int r = i * 4 + srow;
+              if (warp * 32 + r < t.rows) {
+                const uint4 q = ptx::ld_shared_v4(stage + r * 144 + piece * 16);
+                *reinterpret_cast<uint4*>(p.out + (size_t)(t.row0 + warp * 32 + r) * (size_t)p.out_ld + col) = q;
+              }
+            }
+          }
+          __syncwarp();
+        }
+      } else {
+        // ---- GEMM-1 form: SwiGLU of the W1 / W3 halves, 128 output columns
       float sa = 1.f;   // FP8: scale of this thread's row (the gather source row)
       float* s1 = colscale_base + warp * UMMA_N;   // this warp's copy of the W1 / W3 column scales (0 beyond N)
       float* s3 = s1 + 128;
@@ -194,6 +263,7 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
           __syncwarp();
         }
       }
+      }
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(tempty_bar(buf));
@@ -213,14 +283,16 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
           const uint32_t sb = smem_base + s * STAGE_BYTES + A_BYTES;
           ptx::mbar_arrive_expect_tx(full_bar(s), B_BYTES);
           const int k0 = kb * BK_ELEMS;
+          const CUtensorMap* hi_map = PLAIN ? &map_w1 : &map_w3;   // second 128 accumulator columns
+          const int hi_n = PLAIN ? t.n0 + 128 : t.n0;
           if (FP8) {   // K-major boxes of 128 output columns x 128 bytes of K
             ptx::tma_load_3d(sb, &map_w1, full_bar(s), k0, t.n0, t.e);
-            ptx::tma_load_3d(sb + 16384, &map_w3, full_bar(s), k0, t.n0, t.e);
+            ptx::tma_load_3d(sb + 16384, hi_map, full_bar(s), k0, hi_n, t.e);
           } else {     // MN-major slabs of 64 output columns x 64 rows of K
             ptx::tma_load_3d(sb, &map_w1, full_bar(s), t.n0, k0, t.e);
             ptx::tma_load_3d(sb + 8192, &map_w1, full_bar(s), t.n0 + 64, k0, t.e);
-            ptx::tma_load_3d(sb + 16384, &map_w3, full_bar(s), t.n0, k0, t.e);
-            ptx::tma_load_3d(sb + 24576, &map_w3, full_bar(s), t.n0 + 64, k0, t.e);
+            ptx::tma_load_3d(sb + 16384, hi_map, full_bar(s), hi_n, k0, t.e);
+            ptx::tma_load_3d(sb + 24576, hi_map, full_bar(s), hi_n + 64, k0, t.e);
           }
         }
         if (!ok) break;
@@ -275,8 +347,11 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
         const int lr = rbase + 16 * j;
         src[j] = base;
         if (lr < t.rows) {
-          int idx = __ldg(p.gather_idx + t.row0 + lr);
-          if (p.gather_div > 1) idx /= p.gather_div;
+          int idx = t.row0 + lr;   // PLAIN: the rows of h in place
+          if (!PLAIN) {
+            idx = __ldg(p.gather_idx + idx);
+            if (p.gather_div > 1) idx /= p.gather_div;
+          }
           src[j] = base + (size_t)idx * p.a_ld * ELEM;
           live |= 1u << j;
         }
@@ -321,21 +396,32 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
 
 }  // namespace
 
-cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, bool fp8,
-                         cudaStream_t st) {
+namespace {
+template <bool FP8, bool PLAIN>
+cudaError_t launch_form(const GemmParams& p, const CUtensorMap& m_a, const CUtensorMap& m_b, cudaStream_t st) {
   // per device; several host threads may get here at once: setting the attribute twice is harmless
   static std::atomic<bool> attr_set[MAX_DEVICES];
   const int dev = current_device();
   if (!attr_set[dev].load(std::memory_order_acquire)) {
-    cudaError_t e = cudaFuncSetAttribute(ffn_gemm1_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(ffn_gemm1_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm1_kernel<FP8, PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set[dev].store(true, std::memory_order_release);
   }
-  ProfileScope prof(KID_GEMM1, st);
-  if (fp8) return launch_pdl(ffn_gemm1_kernel<true>, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);
-  return launch_pdl(ffn_gemm1_kernel<false>, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, p);
+  ProfileScope prof(PLAIN ? KID_GEMM2 : KID_GEMM1, st);
+  return launch_pdl(ffn_gemm1_kernel<FP8, PLAIN>, sm_count(), THREADS, SMEM_BYTES, st, m_a, m_b, p);
+}
+}  // namespace
+
+cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, bool fp8,
+                         cudaStream_t st) {
+  return fp8 ? launch_form<true, false>(p, m_w1, m_w3, st) : launch_form<false, false>(p, m_w1, m_w3, st);
+}
+
+// GEMM-2 through the single-CTA kernel (128-row tiles): p.a_src = h (or its E4M3 copy), p.a_ld = f,
+// p.tile_prefix = the 128-row tile prefix, p.n_tiles = ceil(N / 256); m_w2 is the weight map.
+cudaError_t launch_gemm2_single(const GemmParams& p, const CUtensorMap& m_w2, bool fp8, cudaStream_t st) {
+  return fp8 ? launch_form<true, true>(p, m_w2, m_w2, st) : launch_form<false, true>(p, m_w2, m_w2, st);
 }
 
 }  // namespace ffn

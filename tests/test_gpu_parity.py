@@ -257,3 +257,13 @@ def test_layer_is_capturable_in_a_cuda_graph():
         torch.cuda.synchronize()
         assert torch.equal(y_graph, y_eager)
     assert run.status()[0] == 0
+
+
+@pytest.mark.parametrize("form", ["pair", "single"])
+def test_both_gemm2_forms_on_the_same_layer(form, monkeypatch):
+    """GEMM-2 has a CTA-pair form (256-row tiles) and a single-CTA form (128-row tiles, taken when experts are
+    small on average); the library picks by shape, TCMOE_GEMM2 forces one.  Both must meet the parity bars on a
+    layer with ragged and empty experts."""
+    monkeypatch.setenv("TCMOE_GEMM2", form)
+    cfg = synth.MoEConfig("g2forms", T=1500, d=320, f=448, E=12, k=3, G=4, bias="zipf", zipf_s=1.3, seed=9)
+    staged(cfg)
