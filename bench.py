@@ -450,11 +450,10 @@ def main():
 
         def step_host(i):
             ln = lanes[i & 1]
-            if fp8:   # no host-buffer entry point for the FP8 layer: the same copies, issued from here
-                with torch.cuda.stream(ln["stream"]):
-                    ln["x_dev"].copy_(x_host, non_blocking=True)
-                    layer(ln["x_dev"], ln["y_dev"], ln["ws"], stream=ln["stream"])
-                    ln["y_host"].copy_(ln["y_dev"], non_blocking=True)
+            if fp8:
+                B.moe_layer_fp8_host(shape, x_host, ln["x_dev"], t["w_gate"], t["bias"], wq["w1"], sc["w1"], wq["w3"],
+                                     sc["w3"], wq["w2"], sc["w2"], ln["y_dev"], ln["y_host"], ln["ws"],
+                                     stream=ln["stream"])
             else:
                 B.moe_layer_host(shape, x_host, ln["x_dev"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"],
                                  ln["y_dev"], ln["y_host"], ln["ws"], stream=ln["stream"])
@@ -522,7 +521,8 @@ def main():
         "e2e": None if e2e_ms is None else
                {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": cfg.T * cfg.d * 2,
                 "d2h_bytes_per_step": cfg.T * cfg.d * 2,
-                "pipeline": "moe_layer_host on 2 alternating streams (double-buffered staging and workspace)"},
+                "pipeline": ("moe_layer_fp8_host" if fp8 else "moe_layer_host") +
+                            " on 2 alternating streams (double-buffered staging and workspace)"},
         "value_two_streams": None if two_stream_ms is None else tokens / (two_stream_ms * 1e-3),
         "gpu_launches": (KERNELS_PER_STEP + (2 if fp8 else 0)) * args.steps,   # FP8: + quantisation of x and of h
         "roofline": {"kernel": "ffn_gemm1_kernel (GEMM-1 + SwiGLU, tcgen05)", "bound": "tensor",

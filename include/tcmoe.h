@@ -207,6 +207,13 @@ int moe_layer_fp8(const moe_shape_t* shape, const void* x, const float* w_gate, 
                   const void* w2q, const float* s2, void* y, float* logits, int32_t* topk_idx, float* topk_w,
                   const moe_layout_t* layout, void* ws, size_t ws_bytes, void* stream);
 
+/* moe_layer_fp8 on HOST activations (bf16 x_host / y_host, pinned for asynchronous copies): the
+ * counterpart of moe_layer_host. */
+int moe_layer_fp8_host(const moe_shape_t* shape, const void* x_host, void* x_dev, const float* w_gate,
+                       const float* logit_bias, int64_t bias_row_stride, const void* w1q, const float* s1,
+                       const void* w3q, const float* s3, const void* w2q, const float* s2, void* y_dev, void* y_host,
+                       void* ws, size_t ws_bytes, void* stream);
+
 /* Dispatch without a workspace (the paper has no counterpart; this entry point exists for
  * callers that cannot supply scratch memory).  Some users of this library run where device
  * memory cannot be obtained around the call: plugins that execute inside a host framework's

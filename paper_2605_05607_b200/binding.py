@@ -36,7 +36,7 @@ MOE_FLAG_COMBINE_IN_EPILOGUE = 2
 EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "moe_status", "moe_strerror",
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",
            "moe_profile_enable", "moe_profile_read", "moe_dispatch_noalloc", "moe_quantize_rows",
-           "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8")
+           "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8", "moe_layer_fp8_host")
 
 
 class MoEShape(ctypes.Structure):
@@ -85,6 +85,7 @@ def lib() -> ctypes.CDLL:
         L.moe_quantize_weights.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp, vp]
         L.moe_expert_ffn_fp8.argtypes = [shp, vp, vp, lay, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.moe_layer_fp8.argtypes = [shp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, lay, vp, sz, vp]
+        L.moe_layer_fp8_host.argtypes = [shp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.moe_profile_enable.argtypes = [ctypes.c_int]
         L.moe_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
         for name in EXPORTS:
@@ -232,6 +233,15 @@ def moe_layer_fp8(shape, x, w_gate, logit_bias, w1q, s1, w3q, s3, w2q, s2, y, ws
                                                 _ptr(y), _ptr(logits), _ptr(topk_idx), _ptr(topk_w),
                                                 ctypes.byref(c) if c is not None else None, _ptr(ws), ws.numel(),
                                                 _stream(stream)))
+
+
+def moe_layer_fp8_host(shape, x_host, x_dev, w_gate, logit_bias, w1q, s1, w3q, s3, w2q, s2, y_dev, y_host, ws,
+                       stream=None) -> None:
+    stride = 0 if logit_bias is None or logit_bias.dim() == 1 else shape.E
+    _check("moe_layer_fp8_host", lib().moe_layer_fp8_host(ctypes.byref(shape), _ptr(x_host), _ptr(x_dev), _ptr(w_gate),
+                                                          _ptr(logit_bias), stride, _ptr(w1q), _ptr(s1), _ptr(w3q),
+                                                          _ptr(s3), _ptr(w2q), _ptr(s2), _ptr(y_dev), _ptr(y_host),
+                                                          _ptr(ws), ws.numel(), _stream(stream)))
 
 
 def moe_combine(shape, o, layout: Layout, topk_idx, topk_w, pg, y, ws, stream=None) -> None:

@@ -515,4 +515,22 @@ int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, co
   return MOE_OK;
 }
 
+int moe_layer_fp8_host(const moe_shape_t* shape, const void* x_host, void* x_dev, const float* w_gate,
+                       const float* logit_bias, int64_t bias_row_stride, const void* w1q, const float* s1,
+                       const void* w3q, const float* s3, const void* w2q, const float* s2, void* y_dev, void* y_host,
+                       void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (x_host == nullptr || x_dev == nullptr || y_dev == nullptr || y_host == nullptr) return MOE_ERR_INVALID_ARG;
+  if (!have_device()) return MOE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t bytes = (size_t)shape->T * shape->d * 2;
+  if (bytes) TCMOE_CUDA(cudaMemcpyAsync(x_dev, x_host, bytes, cudaMemcpyHostToDevice, st));
+  rc = moe_layer_fp8(shape, x_dev, w_gate, logit_bias, bias_row_stride, w1q, s1, w3q, s3, w2q, s2, y_dev, nullptr,
+                     nullptr, nullptr, nullptr, ws, ws_bytes, stream);
+  if (rc != MOE_OK) return rc;
+  if (bytes) TCMOE_CUDA(cudaMemcpyAsync(y_host, y_dev, bytes, cudaMemcpyDeviceToHost, st));
+  return MOE_OK;
+}
+
 }  // extern "C"
