@@ -23,9 +23,12 @@
 // 8-11 % (K = 4096) to 30 % (K = 7168, rows gathered from DRAM) slower; deeper or split A / B
 // rings on that form recovered only part of it and cost a second wait per k-block.
 //
-// A CTA-pair (cta_group::2) variant of this kernel was measured slower: with the UMMA twice as
-// fast per CTA the gather -> arrive -> UMMA chain of the peer CTA no longer fits the pipeline
-// depth, and TMA tile::gather4 sustains only one 4-row instruction per ~40 ns.
+// CTA-pair (cta_group::2) variants of this kernel were measured and not kept.  With lagged
+// publication they lost by 20-60 %; with self-arriving copies (the peer CTA's arrivals relayed to the
+// leader's barrier by one thread, with a RELAXED cluster-scope arrive: a releasing one waits for the
+// copies the SM has in flight and held the kernel at 0.83 us per stage) the paired form reaches the
+// same UMMA rate as this kernel and then loses 4 % to the padding of 256-row tiles.  TMA
+// tile::gather4 as the gather engine sustains only one 4-row instruction per ~40 ns.
 #include "ffn_common.cuh"
 
 #include <atomic>
