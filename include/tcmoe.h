@@ -256,6 +256,18 @@ enum { MOE_KERNEL_TOPK = 1, MOE_KERNEL_MASKS = 2, MOE_KERNEL_FILL = 3, MOE_KERNE
 int moe_profile_enable(int kernel_id);
 int moe_profile_read(float* total_ms, int32_t* launches);
 
+/* Self-test of the bounded waits every kernel of the library relies on (the paper's runtime polls
+ * without a bound, Sec. IV-C; here a wait that outlives its budget ends the kernel with a status
+ * instead of hanging the GPU).  Launches one small kernel that waits, with a budget of `limit_ns`
+ * nanoseconds (1 us .. 100 ms), on a shared-memory barrier that nothing ever signals, with the
+ * same wait routine the GEMM kernels use.  The wait gives up, the kernel records
+ * {MOE_DEV_TIMEOUT, where = MOE_KERNEL_SELFTEST, detail = waited microseconds} in the status block
+ * at `ws` (as every kernel does), sets the abort word and returns normally: the context stays
+ * usable.  moe_status_reset() clears the status afterwards.  Returns MOE_OK once the kernel is
+ * enqueued; read the outcome with moe_status(). */
+enum { MOE_KERNEL_SELFTEST = 9 };
+int moe_selftest_wait_timeout(void* ws, uint64_t limit_ns, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

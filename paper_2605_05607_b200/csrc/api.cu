@@ -2,6 +2,7 @@
 #include "../../include/tcmoe.h"
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -160,9 +161,42 @@ ProfileScope::~ProfileScope() {
 }
 }  // namespace tcmoe
 
+namespace tcmoe {
+namespace {
+// One thread waits on a barrier nobody signals; the bounded wait gives up after `limit_ns`.
+__global__ void selftest_wait_kernel(int32_t* status, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_s;
+  grid_dependency_sync();
+  if (threadIdx.x == 0) {
+    abort_s = 0;
+    ptx::mbar_init(ptx::smem_u32(&bar), 1);
+    ptx::fence_mbar_init();
+    const uint64_t t0 = ptx::globaltimer_ns();
+    volatile int* abort_flag = &abort_s;
+    const bool ok = ptx::mbar_wait<false, 0>(ptx::smem_u32(&bar), 0, abort_flag, abort_flag, limit_ns);
+    if (!ok) {
+      report_error(status, DEV_TIMEOUT, 9, (int)((ptx::globaltimer_ns() - t0) / 1000), blockIdx.x);
+      status[ST_ABORT] = 1;
+    }
+  }
+}
+}  // namespace
+}  // namespace tcmoe
+
 using namespace tcmoe;
 
 extern "C" {
+
+int moe_selftest_wait_timeout(void* ws, uint64_t limit_ns, void* stream) {
+  if (ws == nullptr) return MOE_ERR_INVALID_ARG;
+  if (limit_ns < 1000ull || limit_ns > 100000000ull) return MOE_ERR_INVALID_ARG;
+  if (!aligned(ws, 128)) return MOE_ERR_MISALIGNED;
+  if (!have_device()) return MOE_ERR_CUDA;
+  TCMOE_CUDA(launch_pdl(selftest_wait_kernel, 1, 32, 0, static_cast<cudaStream_t>(stream), static_cast<int32_t*>(ws),
+                        (unsigned long long)limit_ns));
+  return MOE_OK;
+}
 
 int moe_profile_enable(int kernel_id) {
   if (kernel_id < 0 || kernel_id > 8) return MOE_ERR_INVALID_ARG;

@@ -267,3 +267,27 @@ def test_both_gemm2_forms_on_the_same_layer(form, monkeypatch):
     monkeypatch.setenv("TCMOE_GEMM2", form)
     cfg = synth.MoEConfig("g2forms", T=1500, d=320, f=448, E=12, k=3, G=4, bias="zipf", zipf_s=1.3, seed=9)
     staged(cfg)
+
+
+def test_bounded_wait_gives_up_and_the_context_stays_usable():
+    """Every wait in the kernels is bounded: a wait that can never be satisfied ends with a status, not a
+    hang.  The self-test kernel waits on a barrier nothing signals; afterwards the same workspace, once
+    reset, runs the layer as before."""
+    cfg = synth.CONFIGS["C1"]
+    run = H.Run(cfg)
+    run.layer()
+    torch.cuda.synchronize()
+    y_before = run.y.clone()
+    B.moe_selftest_wait_timeout(run.ws, 300_000)            # 300 us budget
+    st = run.status()
+    assert st[0] == B.MOE_DEV_TIMEOUT and st[1] == 9, st
+    assert 300 <= st[2] < 20_000, st                         # waited microseconds: the budget, not much more
+    assert st[4] == 1                                        # abort word: later kernels on this workspace skip their work
+    with pytest.raises(B.MoEError):
+        B.moe_selftest_wait_timeout(run.ws, 10)              # budget below 1 us is refused on the host
+    B.moe_status_reset(run.ws)
+    assert run.status()[0] == 0
+    run.y.zero_()
+    run.layer()
+    torch.cuda.synchronize()
+    assert torch.equal(run.y, y_before) and run.status()[0] == 0
