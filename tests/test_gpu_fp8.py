@@ -106,7 +106,8 @@ def _quantized_weights(t, cfg):
 
 
 @pytest.mark.parametrize("cfg", FP8_CASES, ids=lambda c: c.name)
-@pytest.mark.parametrize("flags", [0, B.MOE_FLAG_COMBINE_IN_EPILOGUE], ids=["combine-kernel", "combine-in-epilogue"])
+@pytest.mark.parametrize("flags", [0, B.MOE_FLAG_COMBINE_IN_EPILOGUE, B.MOE_FLAG_WEIGHT_IN_COMBINE],
+                         ids=["combine-kernel", "combine-in-epilogue", "weight-in-combine"])
 def test_layer_fp8_matches_its_oracle(cfg, flags):
     run = H.Run(cfg, flags)
     t = run.t
@@ -125,7 +126,9 @@ def test_layer_fp8_matches_its_oracle(cfg, flags):
     xq, sx = F.quantize_rows(O.bf16_to_f64(H.bf16_host(t["x"])))
     dt = lay["disp_token"].astype(np.int64)
     ref_w = {n: F.quantize_weights(O.bf16_to_f64(H.bf16_host(t[n]))) for n in ("w1", "w3", "w2")}
-    o_ref = F.expert_ffn_fp8(xq[dt], sx[dt], lay, run.host_w(), *ref_w["w1"], *ref_w["w3"], *ref_w["w2"])
-    _, _, y_ref = O.combine(o_ref, lay, idx_ref, None, cfg.E, cfg.G)
+    in_combine = bool(flags & B.MOE_FLAG_WEIGHT_IN_COMBINE)
+    o_ref = F.expert_ffn_fp8(xq[dt], sx[dt], lay, None if in_combine else run.host_w(), *ref_w["w1"], *ref_w["w3"],
+                             *ref_w["w2"])
+    _, _, y_ref = O.combine(o_ref, lay, idx_ref, run.host_w() if in_combine else None, cfg.E, cfg.G)
     y_gpu = O.bf16_to_f64(H.bf16_host(run.y)[: cfg.T])
     H.assert_close_out(y_gpu, y_ref, "fp8 layer y")
