@@ -256,6 +256,20 @@ enum { MOE_KERNEL_TOPK = 1, MOE_KERNEL_MASKS = 2, MOE_KERNEL_FILL = 3, MOE_KERNE
 int moe_profile_enable(int kernel_id);
 int moe_profile_read(float* total_ms, int32_t* launches);
 
+/* Traffic figures of Sec. II-B / II-C for the routing held in `layout` (a filled dispatch layout
+ * of `shape`), with the G expert groups read as the G GPUs of an expert-parallel node:
+ *   out[0] T   out[1] P = T*k   out[2] N_disp (distinct (token, group) pairs)
+ *   out[3] D = N_disp / T, the mean number of distinct destinations of a token
+ *   out[4] 1 - N_disp / P: share of the point-to-point Dispatch copies that one-copy-per-group
+ *          (in-switch multicast) removes; the same share of Combine rows is removed by the in-group
+ *          pre-reduction
+ *   out[5] (G - D) / D: useless traffic when Dispatch / Combine are emulated by AllGather /
+ *          Reduce-Scatter (the paper's "340 %" for DeepSeek-V3 on 32 GPUs)
+ *   out[6] (D - 1) / (2 D): redundant share of the source <-> switch traffic ("nearly 50 %")
+ *   out[7] 2 D / (1 + D): ideal communication speed-up ("near 2x")
+ * Reads one int32 from the device and synchronises `stream`.  T = 0 gives zeros. */
+int moe_traffic_stats(const moe_shape_t* shape, const moe_layout_t* layout, double out[8], void* stream);
+
 /* Self-test of the bounded waits every kernel of the library relies on (the paper's runtime polls
  * without a bound, Sec. IV-C; here a wait that outlives its budget ends the kernel with a status
  * instead of hanging the GPU).  Launches one small kernel that waits, with a budget of `limit_ns`

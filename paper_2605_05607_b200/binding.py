@@ -36,7 +36,7 @@ MOE_FLAG_COMBINE_IN_EPILOGUE = 2
 EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "moe_status", "moe_strerror",
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",
            "moe_profile_enable", "moe_profile_read", "moe_dispatch_noalloc", "moe_quantize_rows",
-           "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8", "moe_layer_fp8_host", "moe_selftest_wait_timeout")
+           "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8", "moe_layer_fp8_host", "moe_selftest_wait_timeout", "moe_traffic_stats")
 
 
 class MoEShape(ctypes.Structure):
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
         L.moe_layer_fp8.argtypes = [shp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, lay, vp, sz, vp]
         L.moe_layer_fp8_host.argtypes = [shp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.moe_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint64, vp]
+        L.moe_traffic_stats.argtypes = [shp, lay, ctypes.POINTER(ctypes.c_double), vp]
         L.moe_profile_enable.argtypes = [ctypes.c_int]
         L.moe_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
         for name in EXPORTS:
@@ -243,6 +244,14 @@ def moe_layer_fp8_host(shape, x_host, x_dev, w_gate, logit_bias, w1q, s1, w3q, s
                                                           _ptr(logit_bias), stride, _ptr(w1q), _ptr(s1), _ptr(w3q),
                                                           _ptr(s3), _ptr(w2q), _ptr(s2), _ptr(y_dev), _ptr(y_host),
                                                           _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def moe_traffic_stats(shape, layout: Layout, stream=None) -> dict:
+    c = layout.c()
+    out = (ctypes.c_double * 8)()
+    _check("moe_traffic_stats", lib().moe_traffic_stats(ctypes.byref(shape), ctypes.byref(c), out, _stream(stream)))
+    names = ("T", "P", "n_disp", "D", "dedup", "allgather_useless", "redundant_share", "ideal_speedup")
+    return dict(zip(names, list(out)))
 
 
 def moe_selftest_wait_timeout(ws, limit_ns: int, stream=None) -> None:

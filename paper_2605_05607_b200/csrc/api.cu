@@ -188,6 +188,33 @@ using namespace tcmoe;
 
 extern "C" {
 
+int moe_traffic_stats(const moe_shape_t* shape, const moe_layout_t* layout, double out[8], void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (out == nullptr) return MOE_ERR_INVALID_ARG;
+  if ((rc = check_layout(layout)) != MOE_OK) return rc;
+  for (int i = 0; i < 8; ++i) out[i] = 0.0;
+  if (shape->T == 0) return MOE_OK;
+  if (!have_device()) return MOE_ERR_CUDA;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int32_t n_disp = 0;
+  TCMOE_CUDA(cudaMemcpyAsync(&n_disp, layout->group_offsets + shape->G, sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+  TCMOE_CUDA(cudaStreamSynchronize(st));
+  const double T = shape->T, P = (double)shape->T * shape->k, G = shape->G, N = n_disp;
+  const double D = N / T;
+  out[0] = T;
+  out[1] = P;
+  out[2] = N;
+  out[3] = D;
+  out[4] = 1.0 - N / P;
+  if (D > 0.0) {
+    out[5] = (G - D) / D;
+    out[6] = (D - 1.0) / (2.0 * D);
+    out[7] = 2.0 * D / (1.0 + D);
+  }
+  return MOE_OK;
+}
+
 int moe_selftest_wait_timeout(void* ws, uint64_t limit_ns, void* stream) {
   if (ws == nullptr) return MOE_ERR_INVALID_ARG;
   if (limit_ns < 1000ull || limit_ns > 100000000ull) return MOE_ERR_INVALID_ARG;

@@ -291,3 +291,26 @@ def test_bounded_wait_gives_up_and_the_context_stays_usable():
     run.layer()
     torch.cuda.synchronize()
     assert torch.equal(run.y, y_before) and run.status()[0] == 0
+
+
+def test_traffic_stats_match_the_oracle_and_the_papers_printed_figures():
+    """DeepSeek-V3-shaped routing (256 experts, top-8) over 32 groups: the layout's distinct-destination
+    count gives the paper's "340 %" useless AllGather traffic, "nearly 50 %" redundant share and "near 2x"
+    ideal speed-up (Sec. I, II-B, II-C); the same numbers as the oracle's counter."""
+    import json, os
+    cfg = synth.MoEConfig("ds-route", T=8192, d=256, f=64, E=256, k=8, G=32, score_fn=1)
+    run = H.Run(cfg, inputs=synth.make_routing_inputs(cfg, "cuda") | {"w1": None, "w3": None, "w2": None})
+    run.route()
+    run.dispatch()
+    got = B.moe_traffic_stats(run.shape, run.lay)
+    idx_ref, _ = O.route(run.host_logits(), run.host_bias(), cfg.k, cfg.score_fn)
+    D = O.distinct_groups_per_token(idx_ref, cfg.E, cfg.G)
+    ref = O.redundancy_figures(D, cfg.G, cfg.k)
+    assert got["T"] == cfg.T and got["P"] == cfg.P and abs(got["D"] - D) < 1e-12
+    for name in ("allgather_useless", "redundant_share", "ideal_speedup"):
+        assert abs(got[name] - ref[name]) < 1e-12, name
+    assert abs(got["dedup"] - (1 - D / cfg.k)) < 1e-12
+    gold = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "paper_traffic_figures.json")))
+    assert abs(got["allgather_useless"] - gold["allgather_useless_k8"]) <= gold["allgather_useless_tol"]
+    assert gold["redundant_share_min_k8"] <= got["redundant_share"] <= gold["redundant_share_max"]
+    assert gold["ideal_speedup_min_k8"] <= got["ideal_speedup"] <= gold["ideal_speedup_max"]
