@@ -23,9 +23,10 @@ class Slabs:
         return synth.bf16_bits(self.w[int(e)])
 
 
-# C2..C5b: the benchmark configurations; S32 / M16: two of the paper's own evaluation shapes
-# (Small at top-32 of 64 experts, Medium at top-16), 32 groups
-@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5a", "C5b", "S32", "M16"])
+# C2..C5b: the benchmark configurations; S32 / M16 / L32: three of the paper's own evaluation shapes
+# (Small at top-32 of 64 experts, Medium at top-16, Large at top-32: 2^20 expert rows, element
+# offsets beyond 2^32 in o), 32 groups
+@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5a", "C5b", "S32", "M16", "L32"])
 def test_fullsize_layer(name):
     cfg = synth.ALL_CONFIGS[name]
     run = H.Run(cfg)
