@@ -336,7 +336,7 @@ def main():
     ap.add_argument("--impl", default="tcmoe", choices=["tcmoe", "reference"])
     ap.add_argument("--ref-sample", type=int, default=0,
                     help="tokens per step of the reference arm (0: sized from a one-token calibration)")
-    ap.add_argument("--cpu-sample", type=int, default=256, help="tokens of the cpu_baseline leg (0: skip)")
+    ap.add_argument("--cpu-sample", type=int, default=1024, help="tokens of the cpu_baseline leg (0: skip)")
     ap.add_argument("--experts", default="bf16", choices=["bf16", "fp8"],
                     help="bf16 (the benchmark's precision, default) or fp8: E4M3 experts through moe_layer_fp8 "
                          "(per-token / per-output-column scales; gate and combine stay bf16 / fp32)")
