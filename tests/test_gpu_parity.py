@@ -314,3 +314,71 @@ def test_traffic_stats_match_the_oracle_and_the_papers_printed_figures():
     assert abs(got["allgather_useless"] - gold["allgather_useless_k8"]) <= gold["allgather_useless_tol"]
     assert gold["redundant_share_min_k8"] <= got["redundant_share"] <= gold["redundant_share_max"]
     assert gold["ideal_speedup_min_k8"] <= got["ideal_speedup"] <= gold["ideal_speedup_max"]
+
+
+class Guarded:
+    """A tensor carved out of a larger canary-filled allocation: writes before its start or past its end
+    (the memory checker is closed on this machine) show up as damaged canaries."""
+    PAD = 4096
+
+    def __init__(self, numel, dtype, fill=None):
+        esz = torch.empty(0, dtype=dtype).element_size()
+        nbytes = (numel * esz + 127) // 128 * 128
+        self.raw = torch.full((self.PAD + nbytes + self.PAD,), 0xA5, dtype=torch.uint8, device="cuda")
+        self.t = self.raw[self.PAD: self.PAD + numel * esz].view(dtype)
+        self.lo, self.hi = self.PAD, self.PAD + numel * esz
+        if fill is not None:
+            self.t.fill_(fill)
+
+    def intact(self):
+        return bool((self.raw[: self.lo] == 0xA5).all()) and bool((self.raw[self.hi:] == 0xA5).all())
+
+
+@pytest.mark.parametrize("cfg", [
+    synth.MoEConfig("guard-a", T=257, d=136, f=200, E=6, k=3, G=3, seed=5),
+    synth.MoEConfig("guard-b", T=1000, d=272, f=80, E=20, k=5, G=5, bias="zipf", zipf_s=1.5, seed=6),
+    synth.MoEConfig("guard-c", T=130, d=512, f=1024, E=4, k=4, G=2, score_fn=1, seed=7),
+], ids=lambda c: c.name)
+def test_no_entry_point_writes_outside_its_buffers(cfg):
+    """Every output buffer of every entry point sits between canaries (exact sizes, no slack): ragged shapes,
+    partial tiles and K / N tails must not write a byte outside."""
+    t = synth.make_inputs(cfg, "cuda")
+    shape = B.make_shape(cfg)
+    T, E, k, d, P, G = cfg.T, cfg.E, cfg.k, cfg.d, cfg.P, cfg.G
+    g = {
+        "ws": Guarded(B.moe_workspace_bytes(shape), torch.uint8, 0),
+        "logits": Guarded(T * E, torch.float32), "idx": Guarded(P, torch.int32), "w": Guarded(P, torch.float32),
+        "xg": Guarded(T * min(k, G) * d, torch.bfloat16), "o": Guarded(P * d, torch.bfloat16),
+        "y": Guarded(T * d, torch.bfloat16), "pg": Guarded(T * min(k, G) * d, torch.bfloat16),
+        "expert_counts": Guarded(E, torch.int32), "expert_offsets": Guarded(E + 1, torch.int32),
+        "group_counts": Guarded(G, torch.int32), "group_offsets": Guarded(G + 1, torch.int32),
+        "pair_row": Guarded(P, torch.int32), "row_pair": Guarded(P, torch.int32), "al": Guarded(G * T, torch.int32),
+        "disp_token": Guarded(T * min(k, G), torch.int32), "row_src": Guarded(P, torch.int32),
+    }
+    lay = B.Layout(**{n: g[n].t for n in ("expert_counts", "expert_offsets", "group_counts", "group_offsets",
+                                          "pair_row", "row_pair", "al", "disp_token", "row_src")})
+    ws = g["ws"].t
+    xg = g["xg"].t.view(-1, d)
+    o = g["o"].t.view(-1, d)
+    y = g["y"].t.view(-1, d)
+    B.moe_route(shape, t["x"], t["w_gate"], t["bias"], g["logits"].t, g["idx"].t, g["w"].t, ws)
+    B.moe_dispatch(shape, t["x"], g["idx"].t, lay, xg, ws)
+    B.moe_expert_ffn(shape, xg, lay, g["w"].t, t["w1"], t["w3"], t["w2"], o, ws)
+    B.moe_combine(shape, o, lay, g["idx"].t, g["w"].t, g["pg"].t.view(-1, d), y, ws)
+    B.moe_layer(shape, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws, logits=g["logits"].t,
+                topk_idx=g["idx"].t, topk_w=g["w"].t, layout=lay)
+    B.moe_layer(B.make_shape(cfg, B.MOE_FLAG_COMBINE_IN_EPILOGUE), t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"],
+                t["w2"], y, ws)
+    if cfg.d % 16 == 0 and cfg.f % 16 == 0:
+        wq = {n: Guarded(t[n].numel(), torch.uint8) for n in ("w1", "w3", "w2")}
+        sc = {n: Guarded(E * t[n].shape[2], torch.float32) for n in ("w1", "w3", "w2")}
+        for n in wq:
+            B.moe_quantize_weights(t[n], wq[n].t.view(E, t[n].shape[2], t[n].shape[1]), sc[n].t.view(E, -1))
+        B.moe_layer_fp8(shape, t["x"], t["w_gate"], t["bias"], wq["w1"].t, sc["w1"].t, wq["w3"].t, sc["w3"].t,
+                        wq["w2"].t, sc["w2"].t, y, ws)
+        g.update({f"wq_{n}": wq[n] for n in wq})
+        g.update({f"sc_{n}": sc[n] for n in sc})
+    torch.cuda.synchronize()
+    assert B.moe_status(ws)[0] == 0
+    bad = [n for n, buf in g.items() if not buf.intact()]
+    assert not bad, f"canaries damaged around: {bad}"
