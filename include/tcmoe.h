@@ -18,7 +18,8 @@
  *    pointer must be 16-byte aligned; x, xg, o, y, w1, w3, w2 and the workspace
  *    128-byte aligned.
  *  - Calls only enqueue work on `stream` (a cudaStream_t passed as void*) and
- *    never synchronise, except moe_status.  Data-dependent sizes (N_disp,
+ *    never synchronise, except moe_status, moe_traffic_stats and
+ *    moe_profile_read (which return values to the host).  Data-dependent sizes (N_disp,
  *    counts) stay on the device.
  *  - Return value: 0 on success, a negative MOE_ERR_* when the host rejects the
  *    call (nothing is launched then).  Conditions only the device can see go
