@@ -132,3 +132,38 @@ def test_layer_fp8_matches_its_oracle(cfg, flags):
     _, _, y_ref = O.combine(o_ref, lay, idx_ref, run.host_w() if in_combine else None, cfg.E, cfg.G)
     y_gpu = O.bf16_to_f64(H.bf16_host(run.y)[: cfg.T])
     H.assert_close_out(y_gpu, y_ref, "fp8 layer y")
+
+
+def test_fp8_random_shape_sweep():
+    """Seeded sweep over small random shapes for the FP8 layer: ragged T, K and N tails (any multiple of 16),
+    k / G / E combinations, both score functions, all three flag settings."""
+    rng = np.random.default_rng(77)
+    flag_cycle = [0, B.MOE_FLAG_COMBINE_IN_EPILOGUE, B.MOE_FLAG_WEIGHT_IN_COMBINE]
+    for i in range(9):
+        E = int(rng.choice([1, 2, 4, 6, 8, 12, 24]))
+        G = int(rng.choice([g for g in range(1, E + 1) if E % g == 0]))
+        k = int(rng.integers(1, min(E, 5) + 1))
+        cfg = synth.MoEConfig(f"fp8sweep{i}", T=int(rng.integers(1, 400)), d=16 * int(rng.integers(1, 24)),
+                              f=16 * int(rng.integers(1, 24)), E=E, k=k, G=G, score_fn=int(rng.integers(0, 2)),
+                              bias=str(rng.choice(["none", "zipf"])), zipf_s=1.0, seed=300 + i)
+        flags = flag_cycle[i % 3]
+        run = H.Run(cfg, flags)
+        t = run.t
+        wq, sc = _quantized_weights(t, cfg)
+        lay_dev = B.alloc_layout(run.shape)
+        B.moe_layer_fp8(run.shape, t["x"], t["w_gate"], t["bias"], wq["w1"], sc["w1"], wq["w3"], sc["w3"], wq["w2"],
+                        sc["w2"], run.y, run.ws, logits=run.logits, topk_idx=run.idx, topk_w=run.w, layout=lay_dev)
+        torch.cuda.synchronize()
+        assert run.status()[0] == 0, cfg
+        run.lay = lay_dev
+        idx_ref, _ = H.check_route(run)
+        lay = H.check_layout(run, idx_ref)
+        xq, sx = F.quantize_rows(O.bf16_to_f64(H.bf16_host(t["x"])))
+        dt = lay["disp_token"].astype(np.int64)
+        ref_w = {n: F.quantize_weights(O.bf16_to_f64(H.bf16_host(t[n]))) for n in ("w1", "w3", "w2")}
+        in_combine = bool(flags & B.MOE_FLAG_WEIGHT_IN_COMBINE)
+        o_ref = F.expert_ffn_fp8(xq[dt], sx[dt], lay, None if in_combine else run.host_w(), *ref_w["w1"],
+                                 *ref_w["w3"], *ref_w["w2"])
+        _, _, y_ref = O.combine(o_ref, lay, idx_ref, run.host_w() if in_combine else None, cfg.E, cfg.G)
+        y_gpu = O.bf16_to_f64(H.bf16_host(run.y)[: cfg.T])
+        H.assert_close_out(y_gpu, y_ref, f"{cfg}")
