@@ -60,7 +60,7 @@ enum { MOE_SCORE_SOFTMAX = 0,      /* weights = softmax over the k selected keys
        MOE_SCORE_SIGMOID = 1 };    /* weights = sigmoid(key) renormalised over the k      */
 enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1,   /* default (0): gate weight applied in GEMM-2's
                                             epilogue, Combine un-weighted (Sec. III-C)    */
-       MOE_FLAG_COMBINE_IN_EPILOGUE = 2 }; /* moe_layer only: Combine runs inside GEMM-2's
+       MOE_FLAG_COMBINE_IN_EPILOGUE = 2, /* moe_layer only: Combine runs inside GEMM-2's
                                             epilogue (Sec. V, fused pipeline): every weighted
                                             expert row is added into an fp32 accumulator row of
                                             its token with vector reductions, o is never
@@ -71,6 +71,15 @@ enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1,   /* default (0): gate weight applied in 
                                             run-to-run reproducible).  Excludes
                                             MOE_FLAG_WEIGHT_IN_COMBINE; the stage entry points
                                             moe_expert_ffn / moe_combine reject it.        */
+       MOE_FLAG_SPARSE_TOPK = 4 };       /* moe_dispatch / moe_expert_ffn / moe_combine: entries
+                                            of topk_idx may be -1 (slot unused).  The switch of
+                                            Sec. III-D trims a replica to the targets behind its
+                                            port, so a row received by an expert group carries
+                                            between 1 and min(k, m) experts: this is the form of
+                                            its routing table.  expert_offsets[E] is then the
+                                            number of slots in use (<= T*k), pair_row is -1 for
+                                            unused slots, and the per-pair arrays are filled only
+                                            up to expert_offsets[E].                          */
 
 /* Shape of one layer.  Limits: 1 <= k <= min(E, 32); E <= 1024; E % G == 0;
  * d % 8 == 0; f % 8 == 0; T >= 0; T * max(k, G) < 2^31. */

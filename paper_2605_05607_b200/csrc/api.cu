@@ -71,7 +71,8 @@ int check_shape(const moe_shape_t* s) {
   if (s == nullptr) return MOE_ERR_INVALID_ARG;
   if (s->T < 0 || s->d <= 0 || s->f <= 0 || s->E <= 0 || s->k <= 0 || s->G <= 0) return MOE_ERR_INVALID_ARG;
   if (s->score_fn != MOE_SCORE_SOFTMAX && s->score_fn != MOE_SCORE_SIGMOID) return MOE_ERR_INVALID_ARG;
-  if (s->flags & ~(MOE_FLAG_WEIGHT_IN_COMBINE | MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
+  if (s->flags & ~(MOE_FLAG_WEIGHT_IN_COMBINE | MOE_FLAG_COMBINE_IN_EPILOGUE | MOE_FLAG_SPARSE_TOPK))
+    return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_WEIGHT_IN_COMBINE) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
   if (s->k > s->E || s->G > s->E || s->E % s->G != 0) return MOE_ERR_INVALID_ARG;
   if (s->k > 32 || s->E > 1024 || s->d % 8 != 0 || s->f % 8 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
@@ -465,6 +466,7 @@ static int layer_impl(const moe_shape_t* shape, const void* x, const float* w_ga
                       size_t ws_bytes, void* stream) {
   int rc = check_shape(shape);
   if (rc != MOE_OK) return rc;
+  if (shape->flags & MOE_FLAG_SPARSE_TOPK) return MOE_ERR_INVALID_ARG;   // the layer's own top-k fills every slot
   if (fp8 != nullptr) {
     if (shape->d % 16 != 0 || shape->f % 16 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
     if (fp8->s1 == nullptr || fp8->s3 == nullptr || fp8->s2 == nullptr) return MOE_ERR_INVALID_ARG;

@@ -16,7 +16,7 @@ namespace tcmoe {
 // ---- K2a: membership masks -------------------------------------------------------------------
 __global__ void __launch_bounds__(256) build_masks_kernel(const int32_t* __restrict__ topk_idx, uint32_t* emask,
                                                           uint32_t* gmask, int T, int E, int k, int m, int W,
-                                                          int32_t* status) {
+                                                          int32_t* status, int sparse) {
   grid_dependency_sync();
   const int t = blockIdx.x * blockDim.x + threadIdx.x;  // warp w covers tokens 32w .. 32w+31
   const int lane = threadIdx.x & 31;
@@ -25,7 +25,7 @@ __global__ void __launch_bounds__(256) build_masks_kernel(const int32_t* __restr
   for (int j = 0; j < k; ++j) {
     int e = live ? __ldg(topk_idx + (size_t)t * k + j) : -1;
     if (live && (e < 0 || e >= E)) {
-      report_error(status, DEV_INDEX_OUT_OF_RANGE, KID_MASKS, t, e);
+      if (!(sparse && e == -1)) report_error(status, DEV_INDEX_OUT_OF_RANGE, KID_MASKS, t, e);   // -1: unused slot
       e = -1;
     }
     // lanes that picked the same expert (group) fold their bits into one atomicOr
@@ -122,7 +122,10 @@ __global__ void __launch_bounds__(256) fill_layout_kernel(const int32_t* __restr
   }
   for (int j = 0; j < k; ++j) {
     const int e = __ldg(topk_idx + (size_t)t * k + j);
-    if (e < 0 || e >= E) continue;  // already reported by build_masks_kernel
+    if (e < 0 || e >= E) {          // unused slot (sparse top-k), or an index build_masks_kernel reported
+      L.pair_row[(size_t)t * k + j] = -1;
+      continue;
+    }
     const int rank = sc.eprefix[(size_t)e * sc.W + word] + __popc(sc.emask[(size_t)e * sc.W + word] & below);
     const int r = L.expert_offsets[e] + rank;
     const int g = e / m;
@@ -169,7 +172,7 @@ cudaError_t launch_layout(const Shape& s, const int32_t* topk_idx, const Layout&
     return err;  // emask and gmask are adjacent
   const int tb = (s.T + 255) / 256;
   if (s.T > 0 && (err = launch_pdl(build_masks_kernel, tb, 256, 0, st, topk_idx, sc.emask, sc.gmask, s.T, s.E, s.k,
-                                   m, sc.W, status)) != cudaSuccess)
+                                   m, sc.W, status, (s.flags & 4) ? 1 : 0)) != cudaSuccess)
     return err;
   if ((err = launch_pdl(scan_masks_kernel, s.E + s.G, 256, 0, st, sc.emask, sc.gmask, sc.eprefix, sc.gprefix,
                         L.expert_counts, L.group_counts, s.E, sc.W)) != cudaSuccess)
@@ -272,11 +275,15 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
     int my_g = 0x7FFFFFFF, my_row = 0, my_dst = 0;
     float my_w = 1.f;
     if (lane < k) {
-      my_g = __ldg(topk_idx + (size_t)t * k + lane) / m;
-      my_row = __ldg(pair_row + (size_t)t * k + lane);
-      my_dst = __ldg(group_offsets + my_g) + __ldg(al + (size_t)my_g * T + t);
-      if (weighted) my_w = __ldg(topk_w + (size_t)t * k + lane);
+      const int e = __ldg(topk_idx + (size_t)t * k + lane);
+      if (e >= 0) {   // e < 0: unused slot of a sparse top-k table, sorts behind every real slot and is not read
+        my_g = e / m;
+        my_row = __ldg(pair_row + (size_t)t * k + lane);
+        my_dst = __ldg(group_offsets + my_g) + __ldg(al + (size_t)my_g * T + t);
+        if (weighted) my_w = __ldg(topk_w + (size_t)t * k + lane);
+      }
     }
+    const int kv = __popc(__ballot_sync(0xFFFFFFFFu, lane < k && my_g != 0x7FFFFFFF));   // slots in use
     int my_pos = 0;  // number of slots that come before mine
     for (int j = 0; j < k; ++j) {
       const int gj = __shfl_sync(0xFFFFFFFFu, my_g, j);
@@ -290,14 +297,14 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
 #pragma unroll
       for (int q = 0; q < 8; ++q) { total[q] = 0.f; part[q] = 0.f; }
       int prev_dst = -1;
-      for (int s0 = 0; s0 < k; s0 += 8) {
+      for (int s0 = 0; s0 < kv; s0 += 8) {
         uint4 buf[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q)   // all loads of the batch are in flight before the first use
-          if (s0 + q < k) buf[q] = __ldcs(o + (size_t)s_row[wid][s0 + q] * vec_per_row + v);
+          if (s0 + q < kv) buf[q] = __ldcs(o + (size_t)s_row[wid][s0 + q] * vec_per_row + v);
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-          if (s0 + q < k) {
+          if (s0 + q < kv) {
             const int dst = s_dst[wid][s0 + q];
             if (dst != prev_dst && prev_dst >= 0) {   // a group is complete: emit its partial sum
               if (pg != nullptr) pg[(size_t)prev_dst * vec_per_row + v] = pack_bf16x8(part);
@@ -309,7 +316,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
           }
         }
       }
-      if (pg != nullptr) pg[(size_t)prev_dst * vec_per_row + v] = pack_bf16x8(part);
+      if (pg != nullptr && prev_dst >= 0) pg[(size_t)prev_dst * vec_per_row + v] = pack_bf16x8(part);
 #pragma unroll
       for (int c = 0; c < 8; ++c) total[c] += part[c];
       y[(size_t)t * vec_per_row + v] = pack_bf16x8(total);

@@ -382,3 +382,71 @@ def test_no_entry_point_writes_outside_its_buffers(cfg):
     assert B.moe_status(ws)[0] == 0
     bad = [n for n, buf in g.items() if not buf.intact()]
     assert not bad, f"canaries damaged around: {bad}"
+
+
+def test_sparse_topk_tables():
+    """MOE_FLAG_SPARSE_TOPK: slots of topk_idx may be -1 (the routing table of rows received behind one switch
+    port, trimmed to that port's experts).  Layout arrays against a brute-force enumeration written here,
+    outputs against the dense definition restricted to the slots in use."""
+    cfg = synth.MoEConfig("sparse", T=300, d=128, f=192, E=12, k=4, G=3, seed=21)
+    flags = B.MOE_FLAG_SPARSE_TOPK
+    run = H.Run(cfg, flags)
+    run.route()
+    rng = np.random.default_rng(3)
+    idx = run.host_idx().copy()
+    drop = rng.random(idx.shape) < 0.4
+    drop[5] = True                                   # a token with no slot in use at all
+    drop[6] = False
+    idx[drop] = -1
+    run.idx[: cfg.P] = torch.from_numpy(idx.reshape(-1)).cuda()
+    run.dispatch()
+    T, k, E, G, m = cfg.T, cfg.k, cfg.E, cfg.G, cfg.E // cfg.G
+    # brute force: expert-sorted rows by (expert, token); one dispatched row per distinct (token, group)
+    pairs = sorted((int(idx[t, j]), t, j) for t in range(T) for j in range(k) if idx[t, j] >= 0)
+    counts = np.zeros(E, np.int64)
+    for e, _, _ in pairs:
+        counts[e] += 1
+    eoff = np.concatenate([[0], np.cumsum(counts)])
+    pair_row = -np.ones(T * k, np.int64)
+    row_pair = np.array([t * k + j for _, t, j in pairs], np.int64)
+    pair_row[row_pair] = np.arange(len(pairs))
+    touch = sorted({(int(idx[t, j]) // m, t) for t in range(T) for j in range(k) if idx[t, j] >= 0})
+    gcount = np.bincount([g for g, _ in touch], minlength=G)
+    goff = np.concatenate([[0], np.cumsum(gcount)])
+    al = -np.ones((G, T), np.int64)
+    seen = np.zeros(G, np.int64)
+    for g, t in touch:
+        al[g, t] = seen[g]
+        seen[g] += 1
+    L = run.lay
+    npairs = len(pairs)
+    assert np.array_equal(L.expert_counts.cpu().numpy()[:E], counts)
+    assert np.array_equal(L.expert_offsets.cpu().numpy()[: E + 1], eoff) and eoff[-1] == npairs < cfg.P
+    assert np.array_equal(L.pair_row.cpu().numpy()[: T * k], pair_row)
+    assert np.array_equal(L.row_pair.cpu().numpy()[:npairs], row_pair)
+    assert np.array_equal(L.group_offsets.cpu().numpy()[: G + 1], goff)
+    assert np.array_equal(L.al.cpu().numpy()[: G * T].reshape(G, T), al)
+    row_src = np.array([goff[e // m] + al[e // m, t] for e, t, _ in pairs], np.int64)
+    assert np.array_equal(L.row_src.cpu().numpy()[:npairs], row_src)
+    assert run.status()[0] == 0
+    # expert FFN + combine on the sparse table
+    run.ffn()
+    pg = torch.zeros(max(int(goff[-1]), 1), cfg.d, dtype=torch.bfloat16, device="cuda")
+    run.combine(pg)
+    torch.cuda.synchronize()
+    assert run.status()[0] == 0
+    xb = O.bf16_to_f64(H.bf16_host(run.t["x"]))
+    w = run.host_w()
+    wb = {n: H.bf16_host(run.t[n]) for n in ("w1", "w3", "w2")}
+    y_ref = np.zeros((T, cfg.d))
+    for t in range(T):
+        for j in range(k):
+            if idx[t, j] >= 0:
+                e = int(idx[t, j])
+                y_ref[t] += w[t, j] * O.expert_ffn_rows(xb[t:t + 1], wb["w1"][e], wb["w3"][e], wb["w2"][e])[0]
+    y_gpu = O.bf16_to_f64(H.bf16_host(run.y)[:T])
+    H.assert_close_out(y_gpu, y_ref, "sparse y")
+    assert not y_gpu[5].any()                        # no slot in use: the row of y is zero
+    # the flag is refused where the library picks the experts itself
+    with pytest.raises(B.MoEError):
+        run.layer()
