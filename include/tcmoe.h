@@ -266,6 +266,30 @@ enum { MOE_KERNEL_TOPK = 1, MOE_KERNEL_MASKS = 2, MOE_KERNEL_FILL = 3, MOE_KERNE
 int moe_profile_enable(int kernel_id);
 int moe_profile_read(float* total_ms, int32_t* launches);
 
+/* ---- expert parallelism across GPUs (group g = GPU g) -------------------------------------------
+ * The dispatched buffer xg of moe_dispatch is what travels out (segment g to GPU g: one row per
+ * distinct (token, group), Sec. III-D) and one pre-reduced row per (token, group) travels back.
+ * The exchange itself (an all-to-all with the segment sizes group_counts) is the caller's; these
+ * two entry points are the steps expert parallelism adds on either side of it.
+ *
+ * moe_ep_pack: the trimmed target list of every dispatched row (Sec. III-D: a replica is trimmed
+ * to the targets behind its port).  For row n = (t, g), in ascending slot order:
+ *   send_idx[n, 0..kk)  the experts of token t that live in group g, as indices LOCAL to the group
+ *                       (e - g*m), -1 for unused entries;   kk = min(k, m)
+ *   send_w  [n, 0..kk)  their gate weights, 0 for unused entries
+ * Both [T*min(k,G), kk]; segment g of them travels with segment g of xg.  On the receiving GPU the
+ * rows, send_idx and send_w of all senders, concatenated, are x, topk_idx and topk_w of a layer with
+ * shape {T = rows received, E = m, k = kk, G = 1, MOE_FLAG_SPARSE_TOPK}: moe_dispatch (xg = NULL)
+ * builds its layout, moe_expert_ffn runs the local experts on the received rows (row_src is the
+ * identity there), moe_combine sums each received row's outputs - the pre-reduced row that goes back. */
+int moe_ep_pack(const moe_shape_t* shape, const int32_t* topk_idx, const float* topk_w,
+                const moe_layout_t* layout, int32_t* send_idx, float* send_w, void* stream);
+
+/* moe_ep_finish: back [N_disp, d] bf16 holds, in the order of xg, the pre-reduced rows returned by the
+ * GPUs;  y[t] = sum over the groups g that token t touched of back[group_offsets[g] + al[g][t]]
+ * (fp32, ascending g), bf16 out [T, d]. */
+int moe_ep_finish(const moe_shape_t* shape, const void* back, const moe_layout_t* layout, void* y, void* stream);
+
 /* Traffic figures of Sec. II-B / II-C for the routing held in `layout` (a filled dispatch layout
  * of `shape`), with the G expert groups read as the G GPUs of an expert-parallel node:
  *   out[0] T   out[1] P = T*k   out[2] N_disp (distinct (token, group) pairs)

@@ -37,7 +37,7 @@ MOE_FLAG_SPARSE_TOPK = 4
 EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "moe_status", "moe_strerror",
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",
            "moe_profile_enable", "moe_profile_read", "moe_dispatch_noalloc", "moe_quantize_rows",
-           "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8", "moe_layer_fp8_host", "moe_selftest_wait_timeout", "moe_traffic_stats")
+           "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8", "moe_layer_fp8_host", "moe_selftest_wait_timeout", "moe_traffic_stats", "moe_ep_pack", "moe_ep_finish")
 
 
 class MoEShape(ctypes.Structure):
@@ -89,6 +89,8 @@ def lib() -> ctypes.CDLL:
         L.moe_layer_fp8_host.argtypes = [shp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.moe_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint64, vp]
         L.moe_traffic_stats.argtypes = [shp, lay, ctypes.POINTER(ctypes.c_double), vp]
+        L.moe_ep_pack.argtypes = [shp, vp, vp, lay, vp, vp, vp]
+        L.moe_ep_finish.argtypes = [shp, vp, lay, vp, vp]
         L.moe_profile_enable.argtypes = [ctypes.c_int]
         L.moe_profile_read.argtypes = [ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]
         for name in EXPORTS:
@@ -245,6 +247,18 @@ def moe_layer_fp8_host(shape, x_host, x_dev, w_gate, logit_bias, w1q, s1, w3q, s
                                                           _ptr(logit_bias), stride, _ptr(w1q), _ptr(s1), _ptr(w3q),
                                                           _ptr(s3), _ptr(w2q), _ptr(s2), _ptr(y_dev), _ptr(y_host),
                                                           _ptr(ws), ws.numel(), _stream(stream)))
+
+
+def moe_ep_pack(shape, topk_idx, topk_w, layout: Layout, send_idx, send_w, stream=None) -> None:
+    c = layout.c()
+    _check("moe_ep_pack", lib().moe_ep_pack(ctypes.byref(shape), _ptr(topk_idx), _ptr(topk_w), ctypes.byref(c),
+                                            _ptr(send_idx), _ptr(send_w), _stream(stream)))
+
+
+def moe_ep_finish(shape, back, layout: Layout, y, stream=None) -> None:
+    c = layout.c()
+    _check("moe_ep_finish", lib().moe_ep_finish(ctypes.byref(shape), _ptr(back), ctypes.byref(c), _ptr(y),
+                                                _stream(stream)))
 
 
 def moe_traffic_stats(shape, layout: Layout, stream=None) -> dict:

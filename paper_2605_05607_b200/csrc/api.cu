@@ -189,6 +189,31 @@ using namespace tcmoe;
 
 extern "C" {
 
+int moe_ep_pack(const moe_shape_t* shape, const int32_t* topk_idx, const float* topk_w, const moe_layout_t* layout,
+                int32_t* send_idx, float* send_w, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (topk_idx == nullptr || topk_w == nullptr || send_idx == nullptr || send_w == nullptr) return MOE_ERR_INVALID_ARG;
+  if ((rc = check_layout(layout)) != MOE_OK) return rc;
+  if (!aligned(topk_idx, 16) || !aligned(topk_w, 16) || !aligned(send_idx, 16) || !aligned(send_w, 16))
+    return MOE_ERR_MISALIGNED;
+  if (!have_device()) return MOE_ERR_CUDA;
+  TCMOE_CUDA(launch_ep_pack(to_shape(*shape), topk_idx, topk_w, to_layout(*layout), send_idx, send_w,
+                            static_cast<cudaStream_t>(stream)));
+  return MOE_OK;
+}
+
+int moe_ep_finish(const moe_shape_t* shape, const void* back, const moe_layout_t* layout, void* y, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (back == nullptr || y == nullptr) return MOE_ERR_INVALID_ARG;
+  if ((rc = check_layout(layout)) != MOE_OK) return rc;
+  if (!aligned(back, 128) || !aligned(y, 128)) return MOE_ERR_MISALIGNED;
+  if (!have_device()) return MOE_ERR_CUDA;
+  TCMOE_CUDA(launch_ep_finish(to_shape(*shape), back, to_layout(*layout), y, static_cast<cudaStream_t>(stream)));
+  return MOE_OK;
+}
+
 int moe_traffic_stats(const moe_shape_t* shape, const moe_layout_t* layout, double out[8], void* stream) {
   int rc = check_shape(shape);
   if (rc != MOE_OK) return rc;

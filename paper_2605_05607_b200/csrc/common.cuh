@@ -112,6 +112,10 @@ struct Fp8Args {
   float* sh;                  // [P] scratch: row scales of h
 };
 cudaError_t launch_expert_ffn_fp8(const Shape& s, const FfnArgs& a, const Fp8Args& q, cudaStream_t st);
+// ep.cu: the two steps that expert parallelism across GPUs adds to the single-GPU path
+cudaError_t launch_ep_pack(const Shape& s, const int32_t* topk_idx, const float* topk_w, const Layout& L,
+                           int32_t* send_idx, float* send_w, cudaStream_t st);
+cudaError_t launch_ep_finish(const Shape& s, const void* back, const Layout& L, void* y, cudaStream_t st);
 // quant.cu: bf16 -> E4M3 with one scale per row / per (expert, output column)
 cudaError_t launch_quantize_rows(const void* src, long long rows, int cols, void* dst, float* scale, cudaStream_t st);
 cudaError_t launch_quantize_weights(const void* w, int E, int K, int N, void* wq, float* scale, cudaStream_t st);

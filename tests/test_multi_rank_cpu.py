@@ -60,3 +60,46 @@ def test_single_process_helpers():
     a = replicas.make_rank_inputs(CFG, 0, "cpu")
     b = replicas.make_rank_inputs(CFG, 1, "cpu")
     assert torch.equal(a["w2"], b["w2"]) and not torch.equal(a["x"], b["x"])
+
+
+def _ep_exchange_worker(rank, world, port, out):
+    """The exchange of the expert-parallel path with uneven, data-dependent split sizes: every rank sends
+    rank-tagged rows, learns how many it will receive, receives them in sender order, and the return trip
+    brings every row back to where it started."""
+    from paper_2605_05607_b200 import ep
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        send_counts = [3 + rank, 1 + 2 * rank]                      # rows for rank 0, rank 1
+        n = sum(send_counts)
+        rows = (torch.arange(n * 4, dtype=torch.float32).reshape(n, 4) + 1000 * rank)
+        recv_counts = ep.exchange_counts(send_counts)
+        got = ep.all_to_all_rows(rows, send_counts, recv_counts)
+        back = ep.all_to_all_rows(got * 2, recv_counts, send_counts)
+        dist.barrier()
+        out.put((rank, recv_counts, got.tolist(), bool(torch.equal(back, rows * 2))))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_ep_exchange_with_uneven_splits():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_ep_exchange_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    res = {}
+    for _ in range(world):
+        rank, recv_counts, got, round_trip = q.get(timeout=120)
+        res[rank] = (recv_counts, got, round_trip)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    # rank 0 sends 3 rows to rank 0 and 1 to rank 1; rank 1 sends 4 to rank 0 and 3 to rank 1
+    assert res[0][0] == [3, 4] and res[1][0] == [1, 3]
+    r0 = torch.tensor(res[0][1])
+    assert r0.shape == (7, 4) and r0[0, 0] == 0 and r0[3, 0] == 1000        # own rows first, then rank 1's first rows
+    r1 = torch.tensor(res[1][1])
+    assert r1.shape == (4, 4) and r1[0, 0] == 12 and r1[1, 0] == 1000 + 16   # rank 0's 4th row, then rank 1's rows 4..
+    assert res[0][2] and res[1][2]                                           # the return trip restores the order
