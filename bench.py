@@ -340,6 +340,10 @@ def main():
     ap.add_argument("--experts", default="bf16", choices=["bf16", "fp8"],
                     help="bf16 (the benchmark's precision, default) or fp8: E4M3 experts through moe_layer_fp8 "
                          "(per-token / per-output-column scales; gate and combine stay bf16 / fp32)")
+    ap.add_argument("--parallel", default="replicas", choices=["replicas", "ep"],
+                    help="multi-GPU form: replicas (default: weights replicated, tokens sharded, no data-path "
+                         "collective) or ep (expert parallelism: group g on rank g, all-to-all of the dispatched rows "
+                         "and of the pre-reduced rows; needs E % N == 0; bf16 experts)")
     ap.add_argument("--lean", action="store_true",
                     help="timed region only: no e2e / stage / cpu_baseline legs (for profiler captures)")
     ap.add_argument("--stages-only", action="store_true",
@@ -404,6 +408,26 @@ def main():
     def step():
         layer(t["x"], y, ws)
 
+    ep_rank = None
+    if args.parallel == "ep":
+        from paper_2605_05607_b200 import ep
+        assert not fp8 and cfg.E % world == 0 and cfg.bias != "locality", "ep: bf16 experts, E % N == 0, [E] bias only"
+        if dist is None:   # a process group of one rank, so that the same exchange code runs
+            import torch.distributed as dist
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29533")
+            dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", local))
+        cfg = cfg.with_(G=world)
+        sl = slice(rank * cfg.m, (rank + 1) * cfg.m)
+        ep_rank = ep.EpRank(cfg, rank, t["w_gate"], t["bias"], t["w1"][sl].contiguous(), t["w3"][sl].contiguous(),
+                            t["w2"][sl].contiguous())
+        for n in ("w1", "w3", "w2"):
+            t[n] = None                      # only this rank's experts stay resident
+        torch.cuda.empty_cache()
+
+        def step():
+            ep_rank.forward(t["x"])
+
     sampler = None
     if rank == 0:
         sampler = ClockSampler(str(torch.cuda.get_device_properties(local).uuid))
@@ -434,9 +458,11 @@ def main():
     elapsed_ms = replicas.max_over_ranks(elapsed_ms, dist, "cuda")
     status = B.moe_status(ws)
     assert status[0] == 0, f"device status {status}"
+    if ep_rank is not None:
+        assert all(c == 0 for c in ep_rank.status()), ep_rank.status()
 
     e2e_ms = two_stream_ms = None
-    if not args.lean:
+    if not args.lean and ep_rank is None:
         # ---- end to end through the host-buffer entry point: every step copies its x from pinned
         # host memory and reads its y back.  Two streams with their own staging buffers and
         # workspaces alternate between steps, so the copies of one step overlap the kernels of the
@@ -524,7 +550,9 @@ def main():
                 "pipeline": ("moe_layer_fp8_host" if fp8 else "moe_layer_host") +
                             " on 2 alternating streams (double-buffered staging and workspace)"},
         "value_two_streams": None if two_stream_ms is None else tokens / (two_stream_ms * 1e-3),
-        "gpu_launches": (KERNELS_PER_STEP + (2 if fp8 else 0)) * args.steps,   # FP8: + quantisation of x and of h
+        # FP8: + quantisation of x and of h; ep: route 3, dispatch 5, pack 1, receiver layout 4 + tile prefix 1 + 2 GEMMs +
+        # combine 1, finish 1
+        "gpu_launches": (18 if ep_rank is not None else KERNELS_PER_STEP + (2 if fp8 else 0)) * args.steps,
         "roofline": {"kernel": "ffn_gemm1_kernel (GEMM-1 + SwiGLU, tcgen05)", "bound": "tensor",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": (achieved / peak) if achieved else None,
@@ -537,11 +565,15 @@ def main():
                          "(geomean 1.59x) on a SIMULATED 32-GPU GH200 NVL32 (BookSim2 + Accel-Sim, H200-configured "
                          "GPUs, NVLink 4, FP8 GEMMs); no tokens/s, GB/s or TFLOP/s for this path, hence vs_baseline null",
     }
+    if ep_rank is not None:
+        line["config"]["parallelism"] = (f"expert parallel x{world}: {cfg.m} experts per GPU, all-to-all of one row per "
+                                         "(token, group) out and one pre-reduced row back; split sizes read back once per layer")
+        line["stages"] = None
     if fp8:
         line["experts"] = ("E4M3 weights and activations, one fp32 scale per token / per (expert, output column), "
                            "fp32 accumulation; a reduced-precision variant, not the benchmark's bf16 configuration")
         del wq, sc
-    if world == 1 and not args.lean:
+    if world == 1 and not args.lean and ep_rank is None:
         line["stages"] = stage_breakdown(cfg, t)
     if world == 1 and args.report and not args.lean:
         report = {cfg.name: line["stages"]}
@@ -556,7 +588,7 @@ def main():
         os.makedirs(os.path.dirname(os.path.abspath(args.report)), exist_ok=True)
         json.dump({"peaks": pk, "configs": report}, open(args.report, "w"), indent=1)
         t = synth.make_inputs(cfg, "cuda") if args.cpu_sample > 0 else None
-    if world == 1 and args.cpu_sample > 0 and not args.lean:
+    if world == 1 and args.cpu_sample > 0 and not args.lean and ep_rank is None:
         dt, n = oracle_sample_run(cfg, t, args.cpu_sample)
         line["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                                 "sample": f"{n} of {cfg.T} tokens, {dt:.1f} s (gate + top-k + expert FFN + combine)"}

@@ -75,3 +75,30 @@ def test_ep_pack_lists_are_the_trimmed_targets():
         assert 1 <= len(want) <= kk
         assert got_i[n, : len(want)].tolist() == [e for e, _ in want] and (got_i[n, len(want):] == -1).all()
         assert np.array_equal(got_w[n, : len(want)], np.float32([x for _, x in want])) and not got_w[n, len(want):].any()
+
+
+def test_forward_over_nccl_with_one_rank():
+    """EpRank.forward with a real NCCL process group of size 1 (all this box offers): the exchange degenerates
+    to a copy, everything else is the code path several GPUs would run."""
+    import os
+    import socket
+    import torch.distributed as dist
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK="0", WORLD_SIZE="1")
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", 0))
+    try:
+        cfg = synth.MoEConfig("ep-nccl1", T=300, d=128, f=192, E=6, k=3, G=1, seed=51)
+        t = synth.make_inputs(cfg, "cuda")
+        rank = ep.EpRank(cfg, 0, t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"])
+        y = rank.forward(t["x"]).clone()
+        torch.cuda.synchronize()
+        assert all(c == 0 for c in rank.status())
+        run = H.Run(cfg, inputs=t)
+        run.layer()
+        torch.cuda.synchronize()
+        mx, mean = H.out_errors(O.bf16_to_f64(H.bf16_host(y)), O.bf16_to_f64(H.bf16_host(run.y)[: cfg.T]))
+        assert mx <= 1e-2 and mean <= 3e-3, (mx, mean)
+    finally:
+        dist.destroy_process_group()
