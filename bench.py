@@ -252,11 +252,18 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
     def layer_epilogue_combine():
         B.moe_layer(shape_epi, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws)
 
-    seq_ms, fus_ms, epi_ms = [], [], []
+    # fourth variant: GEMM-1 and GEMM-2 as one persistent kernel paced by the 128-row tile tracker
+    shape_trk = B.make_shape(cfg, B.MOE_FLAG_FUSED_FFN)
+
+    def layer_single_kernel_ffn():
+        B.moe_layer(shape_trk, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws)
+
+    seq_ms, fus_ms, epi_ms, trk_ms = [], [], [], []
     for _ in range(reps):
         seq_ms.append(timed(unfused_seq))
         fus_ms.append(timed(calls["layer_fused"]))
         epi_ms.append(timed(layer_epilogue_combine))
+        trk_ms.append(timed(layer_single_kernel_ffn))
     # in-layer (back to back, no idle gap) kernel times of the fused call
     for kn in kernels["layer_fused"]:
         B.moe_profile_enable(B.KERNEL_IDS[kn])
@@ -302,6 +309,7 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
     out["summary"] = {"unfused_sum_ms": unfused, "unfused_back_to_back_ms": float(np.median(seq_ms)),
                       "fused_back_to_back_ms": float(np.median(fus_ms)),
                       "fused_epilogue_combine_back_to_back_ms": float(np.median(epi_ms)),
+                      "fused_single_kernel_ffn_back_to_back_ms": float(np.median(trk_ms)),
                       "fused_ms": out["layer_fused"]["ms"],
                       "fused_tokens_per_s": T / out["layer_fused"]["ms"] * 1e3,
                       "n_disp": n_disp, "pairs": P, "dedup": 1.0 - n_disp / P,

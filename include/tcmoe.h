@@ -71,7 +71,7 @@ enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1,   /* default (0): gate weight applied in 
                                             run-to-run reproducible).  Excludes
                                             MOE_FLAG_WEIGHT_IN_COMBINE; the stage entry points
                                             moe_expert_ffn / moe_combine reject it.        */
-       MOE_FLAG_SPARSE_TOPK = 4 };       /* moe_dispatch / moe_expert_ffn / moe_combine: entries
+       MOE_FLAG_SPARSE_TOPK = 4,         /* moe_dispatch / moe_expert_ffn / moe_combine: entries
                                             of topk_idx may be -1 (slot unused).  The switch of
                                             Sec. III-D trims a replica to the targets behind its
                                             port, so a row received by an expert group carries
@@ -80,6 +80,13 @@ enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1,   /* default (0): gate weight applied in 
                                             number of slots in use (<= T*k), pair_row is -1 for
                                             unused slots, and the per-pair arrays are filled only
                                             up to expert_offsets[E].                          */
+       MOE_FLAG_FUSED_FFN = 8 };         /* moe_expert_ffn / moe_layer (bf16 experts): GEMM-1 and
+                                            GEMM-2 run as ONE persistent kernel paced by a tile
+                                            tracker (Sec. IV token-centric kernel fusion, tiles of
+                                            128 tokens): a GEMM-2 tile starts as soon as the
+                                            128 rows of h it reads are complete.  Same results as
+                                            the two-kernel form (bit for bit); excludes
+                                            MOE_FLAG_COMBINE_IN_EPILOGUE.                      */
 
 /* Shape of one layer.  Limits: 1 <= k <= min(E, 32); E <= 1024; E % G == 0;
  * d % 8 == 0; f % 8 == 0; T >= 0; T * max(k, G) < 2^31. */

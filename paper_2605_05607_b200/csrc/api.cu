@@ -15,7 +15,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Regions of the workspace, in order.  Every region starts on a 1 KiB boundary.
 struct WsPlan {
-  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, wsplit, h, hq, sh, xq, sx, o, logits, topk_idx, topk_w;
+  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, blk_start, blk_info, n_blocks, done, wsplit, h, hq, sh, xq, sx, o, logits, topk_idx, topk_w;
   size_t expert_counts, expert_offsets, group_counts, group_offsets, pair_row, row_pair, al, disp_token, row_src;
   size_t total;
   int W;
@@ -43,6 +43,13 @@ WsPlan plan(const moe_shape_t& s) {
   p.gprefix = take(G * W * 4);
   p.mt_prefix = take((E + 1) * 4);
   p.mp_prefix = take((E + 1) * 4);
+  {   // single-kernel FFN: task tables and tile tracker
+    const size_t nbmax = fused_table_blocks(Shape{s.T, s.d, s.f, s.E, s.k, s.G, s.score_fn, s.flags});
+    p.blk_start = take((nbmax + 1) * 4);
+    p.blk_info = take(nbmax * 16);
+    p.n_blocks = take(4);
+    p.done = take((P / 128 + E + 1) * 4);
+  }
   p.wsplit = take(gate_split_bytes(s.d, s.E));
   p.h = take(P * (size_t)s.f * 2);
   p.hq = take(P * (size_t)s.f);   // FP8 form: E4M3 copy of h and its row scales
@@ -71,8 +78,9 @@ int check_shape(const moe_shape_t* s) {
   if (s == nullptr) return MOE_ERR_INVALID_ARG;
   if (s->T < 0 || s->d <= 0 || s->f <= 0 || s->E <= 0 || s->k <= 0 || s->G <= 0) return MOE_ERR_INVALID_ARG;
   if (s->score_fn != MOE_SCORE_SOFTMAX && s->score_fn != MOE_SCORE_SIGMOID) return MOE_ERR_INVALID_ARG;
-  if (s->flags & ~(MOE_FLAG_WEIGHT_IN_COMBINE | MOE_FLAG_COMBINE_IN_EPILOGUE | MOE_FLAG_SPARSE_TOPK))
+  if (s->flags & ~(MOE_FLAG_WEIGHT_IN_COMBINE | MOE_FLAG_COMBINE_IN_EPILOGUE | MOE_FLAG_SPARSE_TOPK | MOE_FLAG_FUSED_FFN))
     return MOE_ERR_INVALID_ARG;
+  if ((s->flags & MOE_FLAG_FUSED_FFN) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_WEIGHT_IN_COMBINE) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
   if (s->k > s->E || s->G > s->E || s->E % s->G != 0) return MOE_ERR_INVALID_ARG;
   if (s->k > 32 || s->E > 1024 || s->d % 8 != 0 || s->f % 8 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
@@ -393,8 +401,13 @@ int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t*
   a.topk_w = in_combine ? nullptr : topk_w;
   a.row_pair = layout->row_pair;
   a.expert_offsets = layout->expert_offsets;
+  a.expert_counts = layout->expert_counts;
   a.mt_prefix = at<int32_t>(ws, p.mt_prefix);
   a.mp_prefix = at<int32_t>(ws, p.mp_prefix);
+  a.blk_start = at<int32_t>(ws, p.blk_start);
+  a.blk_info = at<void>(ws, p.blk_info);
+  a.n_blocks = at<int32_t>(ws, p.n_blocks);
+  a.done = at<int32_t>(ws, p.done);
   a.status = at<int32_t>(ws, p.status);
   // rebuilt from the counts so that this call does not depend on what moe_dispatch left in ws
   TCMOE_CUDA(launch_tile_prefix(to_shape(*shape), layout->expert_counts, at<int32_t>(ws, p.mt_prefix),
@@ -428,6 +441,7 @@ int moe_expert_ffn_fp8(const moe_shape_t* shape, const void* xq, const float* sx
   int rc = check_shape(shape);
   if (rc != MOE_OK) return rc;
   if (shape->d % 16 != 0 || shape->f % 16 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;   // 16-byte rows of 8-bit elements
+  if (shape->flags & MOE_FLAG_FUSED_FFN) return MOE_ERR_INVALID_ARG;                  // bf16 experts only
   if (xq == nullptr || sx == nullptr || w1q == nullptr || w3q == nullptr || w2q == nullptr || s1 == nullptr ||
       s3 == nullptr || s2 == nullptr || o == nullptr)
     return MOE_ERR_INVALID_ARG;
@@ -453,8 +467,13 @@ int moe_expert_ffn_fp8(const moe_shape_t* shape, const void* xq, const float* sx
   a.topk_w = in_combine ? nullptr : topk_w;
   a.row_pair = layout->row_pair;
   a.expert_offsets = layout->expert_offsets;
+  a.expert_counts = layout->expert_counts;
   a.mt_prefix = at<int32_t>(ws, p.mt_prefix);
   a.mp_prefix = at<int32_t>(ws, p.mp_prefix);
+  a.blk_start = at<int32_t>(ws, p.blk_start);
+  a.blk_info = at<void>(ws, p.blk_info);
+  a.n_blocks = at<int32_t>(ws, p.n_blocks);
+  a.done = at<int32_t>(ws, p.done);
   a.status = at<int32_t>(ws, p.status);
   Fp8Args q{sx, s1, s3, s2, at<void>(ws, p.hq), at<float>(ws, p.sh)};
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -493,6 +512,7 @@ static int layer_impl(const moe_shape_t* shape, const void* x, const float* w_ga
   if (rc != MOE_OK) return rc;
   if (shape->flags & MOE_FLAG_SPARSE_TOPK) return MOE_ERR_INVALID_ARG;   // the layer's own top-k fills every slot
   if (fp8 != nullptr) {
+    if (shape->flags & MOE_FLAG_FUSED_FFN) return MOE_ERR_INVALID_ARG;   // bf16 experts only
     if (shape->d % 16 != 0 || shape->f % 16 != 0) return MOE_ERR_UNSUPPORTED_SHAPE;
     if (fp8->s1 == nullptr || fp8->s3 == nullptr || fp8->s2 == nullptr) return MOE_ERR_INVALID_ARG;
     if (!aligned(fp8->s1, 4) || !aligned(fp8->s3, 4) || !aligned(fp8->s2, 4)) return MOE_ERR_MISALIGNED;
@@ -551,8 +571,13 @@ static int layer_impl(const moe_shape_t* shape, const void* x, const float* w_ga
   a.topk_w = (s.flags & MOE_FLAG_WEIGHT_IN_COMBINE) ? nullptr : tw;
   a.row_pair = L.row_pair;
   a.expert_offsets = L.expert_offsets;
+  a.expert_counts = L.expert_counts;
   a.mt_prefix = at<int32_t>(ws, p.mt_prefix);
   a.mp_prefix = at<int32_t>(ws, p.mp_prefix);
+  a.blk_start = at<int32_t>(ws, p.blk_start);
+  a.blk_info = at<void>(ws, p.blk_info);
+  a.n_blocks = at<int32_t>(ws, p.n_blocks);
+  a.done = at<int32_t>(ws, p.done);
   a.status = status;
   if (s.flags & MOE_FLAG_COMBINE_IN_EPILOGUE) {
     // o never materialises: GEMM-2 adds each weighted row into its token's fp32 accumulator

@@ -101,8 +101,15 @@ struct FfnArgs {
   const int32_t* expert_offsets;
   const int32_t* mt_prefix;   // 128-row tiles per expert, exclusive prefix
   const int32_t* mp_prefix;   // 256-row pair tiles per expert, exclusive prefix
+  // single-kernel FFN (MOE_FLAG_FUSED_FFN): task tables and the tile tracker, scratch in the workspace
+  const int32_t* expert_counts;
+  int32_t* blk_start;
+  void* blk_info;
+  int32_t* n_blocks;
+  int32_t* done;
   int32_t* status;
 };
+size_t fused_table_blocks(const Shape& s);   // task-block capacity for a shape (ffn_fused.cu)
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st);
 // FP8 form of the expert FFN: a.a_src / a.w1 / a.w3 / a.w2 hold E4M3 codes (weights [E, N, K]).
 struct Fp8Args {

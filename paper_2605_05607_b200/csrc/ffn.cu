@@ -112,8 +112,43 @@ static bool small_experts(const Shape& s) {
   return (long long)s.T * s.k < 512ll * s.E;
 }
 
+size_t fused_table_blocks(const Shape& s) { return ffn::fused_max_blocks(s.T, s.k, s.E); }
+
+// flag bit 8 (MOE_FLAG_FUSED_FFN): both GEMMs in one persistent kernel paced by the tile tracker
+static cudaError_t launch_expert_ffn_fused(const Shape& s, const FfnArgs& a, cudaStream_t st) {
+  CUtensorMap m_w1, m_w3, m_w2;
+  if (!make_weight_map(&m_w1, a.w1, s.E, s.d, s.f) || !make_weight_map(&m_w3, a.w3, s.E, s.d, s.f) ||
+      !make_weight_map(&m_w2, a.w2, s.E, s.f, s.d))
+    return cudaErrorInvalidValue;
+  ffn::FusedParams p{};
+  p.x = a.a_src;
+  p.x_ld = s.d;
+  p.gather_idx = a.gather_idx;
+  p.gather_div = a.gather_div;
+  p.h = static_cast<__nv_bfloat16*>(a.h);
+  p.o = static_cast<__nv_bfloat16*>(a.o);
+  p.topk_w = a.topk_w;
+  p.row_pair = a.row_pair;
+  p.expert_offsets = a.expert_offsets;
+  p.mt_prefix = a.mt_prefix;
+  p.blk_start = a.blk_start;
+  p.blk_info = static_cast<const int4*>(a.blk_info);
+  p.n_blocks = a.n_blocks;
+  p.done = a.done;
+  p.E = s.E;
+  p.d = s.d;
+  p.f = s.f;
+  p.n1 = (s.f + 127) / 128;
+  p.n2 = (s.d + 255) / 256;
+  p.status = a.status;
+  const size_t done_entries = (size_t)s.T * s.k / ffn::BM + s.E + 1;
+  return ffn::launch_ffn_fused(p, a.expert_counts, a.blk_start, static_cast<int4*>(a.blk_info), a.n_blocks,
+                               done_entries, m_w1, m_w3, m_w2, st);
+}
+
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st) {
   if (s.T == 0) return cudaSuccess;
+  if ((s.flags & 8) && a.y_acc == nullptr && a.blk_start != nullptr) return launch_expert_ffn_fused(s, a, st);
   const int P = s.T * s.k;
   CUtensorMap m_w1, m_w3, m_w2, m_h;
   if (!make_weight_map(&m_w1, a.w1, s.E, s.d, s.f) || !make_weight_map(&m_w3, a.w3, s.E, s.d, s.f) ||

@@ -103,6 +103,26 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Parameters of the single-kernel FFN (ffn_fused.cu)
+struct FusedParams {
+  const void* x;                // GEMM-1 gather source (xg or x), bf16
+  int x_ld;
+  const int32_t* gather_idx;
+  int gather_div;
+  __nv_bfloat16* h;             // [P, f] intermediate
+  __nv_bfloat16* o;             // [P, d] out
+  const float* topk_w;          // GEMM-2 epilogue weights (NULL: 1)
+  const int32_t* row_pair;
+  const int32_t* expert_offsets;
+  const int32_t* mt_prefix;     // [E+1] 128-row tile prefix: tracker slot base per expert
+  const int32_t* blk_start;     // [n_blocks + 1] cumulative task counts of the task blocks
+  const int4* blk_info;         // [n_blocks] {0: GEMM-1 / 1: GEMM-2, expert, first row tile, row tiles}
+  const int32_t* n_blocks;      // device scalar
+  int32_t* done;                // tracker: parts stored per 128-row tile of h (zeroed before the launch)
+  int E, d, f, n1, n2;          // n1 = ceil(f / 128) GEMM-1 column tiles, n2 = ceil(d / 256) GEMM-2 column tiles
+  int32_t* status;
+};
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -113,6 +133,10 @@ cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUt
                          cudaStream_t st);
 cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, bool fp8,
                          cudaStream_t st);
+size_t fused_max_blocks(int T, int k, int E);   // capacity of blk_start (+1) / blk_info for a shape
+cudaError_t launch_ffn_fused(const FusedParams& p, const int32_t* expert_counts, int32_t* blk_start, int4* blk_info,
+                             int32_t* n_blocks, size_t done_entries, const CUtensorMap& m_w1, const CUtensorMap& m_w3,
+                             const CUtensorMap& m_w2, cudaStream_t st);
 // GEMM-2 on 128-row single-CTA tiles (small experts): p.a_src / p.a_ld = h rows, no Combine-in-epilogue form
 cudaError_t launch_gemm2_single(const GemmParams& p, const CUtensorMap& m_w2, bool fp8, cudaStream_t st);
 

@@ -450,3 +450,34 @@ def test_sparse_topk_tables():
     # the flag is refused where the library picks the experts itself
     with pytest.raises(B.MoEError):
         run.layer()
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
+def test_single_kernel_ffn_with_tile_tracker(cfg):
+    """MOE_FLAG_FUSED_FFN: GEMM-1 and GEMM-2 as one persistent kernel paced by the 128-row tile tracker.  The
+    expert outputs must equal the two-kernel form bit for bit (same operands, same accumulation order per
+    element), in the staged entry point and in the fused layer, twice in a row (the tracker is cleared by every
+    call)."""
+    if "wcombine" in cfg.name:
+        pytest.skip("covered by the default-weight cases")
+    run = H.Run(cfg)
+    run.route()
+    run.dispatch()
+    run.ffn()
+    o_two = run.o.clone()
+    run.layer()
+    y_two = run.y.clone()
+    fused = H.Run(cfg, B.MOE_FLAG_FUSED_FFN, inputs=run.t)
+    fused.route()
+    fused.dispatch()
+    for _ in range(2):
+        fused.o.fill_(7.0)
+        fused.ffn()
+        torch.cuda.synchronize()
+        assert fused.status()[0] == 0, fused.status()
+        assert torch.equal(fused.o[: cfg.P], o_two[: cfg.P])
+        fused.y.fill_(7.0)
+        fused.layer()
+        torch.cuda.synchronize()
+        assert fused.status()[0] == 0
+        assert torch.equal(fused.y[: cfg.T], y_two[: cfg.T])
