@@ -153,3 +153,22 @@ def test_fullsize_layer_fp8(name):
     y_gpu = O.bf16_to_f64(H.bf16_host(run.y[torch.from_numpy(toks).cuda()]))
     tol = 2.0 ** -8 * np.abs(y_ref) + 2.0 ** -22 * np.abs(y_ref).max() + 1e-30
     assert np.all(np.abs(y_gpu - y_ref) <= tol), f"{name} fp8 combine"
+
+
+@pytest.mark.parametrize("name", ["C4", "C3"])
+def test_fullsize_single_kernel_ffn_equals_two_kernels(name):
+    """MOE_FLAG_FUSED_FFN at full size (C4: 131 072 expert rows in 1 024-row experts; C3: Zipf-skewed, empty and
+    tiny experts): the tracker-paced single kernel writes the same o, bit for bit, as GEMM-1 followed by GEMM-2."""
+    cfg = synth.ALL_CONFIGS[name]
+    run = H.Run(cfg)
+    run.route()
+    run.dispatch()
+    run.ffn()
+    o_two = run.o.clone()
+    fused = H.Run(cfg, B.MOE_FLAG_FUSED_FFN, inputs=run.t)
+    fused.idx, fused.w, fused.lay, fused.xg = run.idx, run.w, run.lay, run.xg
+    fused.o.fill_(3.0)
+    fused.ffn()
+    torch.cuda.synchronize()
+    assert fused.status()[0] == 0
+    assert torch.equal(fused.o[: cfg.P], o_two[: cfg.P])
