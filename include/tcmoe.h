@@ -80,6 +80,11 @@ enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1,   /* default (0): gate weight applied in 
                                             number of slots in use (<= T*k), pair_row is -1 for
                                             unused slots, and the per-pair arrays are filled only
                                             up to expert_offsets[E].                          */
+       MOE_FLAG_SM_PARTITION = 16,       /* with MOE_FLAG_FUSED_FFN: the thread blocks are divided
+                                            between the stages as in Sec. IV - two thirds of the
+                                            SMs take only GEMM-1 tiles, one third only GEMM-2
+                                            tiles, the second group paced by the tracker alone.
+                                            Same results.                                      */
        MOE_FLAG_FUSED_FFN = 8 };         /* moe_expert_ffn / moe_layer (bf16 experts): GEMM-1 and
                                             GEMM-2 run as ONE persistent kernel paced by a tile
                                             tracker (Sec. IV token-centric kernel fusion, tiles of

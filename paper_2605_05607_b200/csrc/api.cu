@@ -45,9 +45,9 @@ WsPlan plan(const moe_shape_t& s) {
   p.mp_prefix = take((E + 1) * 4);
   {   // single-kernel FFN: task tables and tile tracker
     const size_t nbmax = fused_table_blocks(Shape{s.T, s.d, s.f, s.E, s.k, s.G, s.score_fn, s.flags});
-    p.blk_start = take((nbmax + 1) * 4);
-    p.blk_info = take(nbmax * 16);
-    p.n_blocks = take(4);
+    p.blk_start = take(3 * (nbmax + 1) * 4);   // interleaved | GEMM-1 only | GEMM-2 only
+    p.blk_info = take(3 * (nbmax + 1) * 16);
+    p.n_blocks = take(3 * 4);
     p.done = take((P / 128 + E + 1) * 4);
   }
   p.wsplit = take(gate_split_bytes(s.d, s.E));
@@ -78,8 +78,10 @@ int check_shape(const moe_shape_t* s) {
   if (s == nullptr) return MOE_ERR_INVALID_ARG;
   if (s->T < 0 || s->d <= 0 || s->f <= 0 || s->E <= 0 || s->k <= 0 || s->G <= 0) return MOE_ERR_INVALID_ARG;
   if (s->score_fn != MOE_SCORE_SOFTMAX && s->score_fn != MOE_SCORE_SIGMOID) return MOE_ERR_INVALID_ARG;
-  if (s->flags & ~(MOE_FLAG_WEIGHT_IN_COMBINE | MOE_FLAG_COMBINE_IN_EPILOGUE | MOE_FLAG_SPARSE_TOPK | MOE_FLAG_FUSED_FFN))
+  if (s->flags & ~(MOE_FLAG_WEIGHT_IN_COMBINE | MOE_FLAG_COMBINE_IN_EPILOGUE | MOE_FLAG_SPARSE_TOPK | MOE_FLAG_FUSED_FFN |
+                   MOE_FLAG_SM_PARTITION))
     return MOE_ERR_INVALID_ARG;
+  if ((s->flags & MOE_FLAG_SM_PARTITION) && !(s->flags & MOE_FLAG_FUSED_FFN)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_FUSED_FFN) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_WEIGHT_IN_COMBINE) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
   if (s->k > s->E || s->G > s->E || s->E % s->G != 0) return MOE_ERR_INVALID_ARG;

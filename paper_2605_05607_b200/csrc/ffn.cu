@@ -134,6 +134,9 @@ static cudaError_t launch_expert_ffn_fused(const Shape& s, const FfnArgs& a, cud
   p.blk_start = a.blk_start;
   p.blk_info = static_cast<const int4*>(a.blk_info);
   p.n_blocks = a.n_blocks;
+  p.tbl_stride = (int)fused_table_blocks(s) + 1;
+  // flag bit 16 (MOE_FLAG_SM_PARTITION): two thirds of the SMs for GEMM-1 (it has two thirds of the flops)
+  p.part_g1 = (s.flags & 16) ? (2 * sm_count() + 1) / 3 : 0;
   p.done = a.done;
   p.E = s.E;
   p.d = s.d;

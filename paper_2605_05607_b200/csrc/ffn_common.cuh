@@ -115,9 +115,12 @@ struct FusedParams {
   const int32_t* row_pair;
   const int32_t* expert_offsets;
   const int32_t* mt_prefix;     // [E+1] 128-row tile prefix: tracker slot base per expert
-  const int32_t* blk_start;     // [n_blocks + 1] cumulative task counts of the task blocks
-  const int4* blk_info;         // [n_blocks] {0: GEMM-1 / 1: GEMM-2, expert, first row tile, row tiles}
-  const int32_t* n_blocks;      // device scalar
+  // three task tables `tbl_stride` entries apart: interleaved, GEMM-1 blocks alone, GEMM-2 blocks alone
+  const int32_t* blk_start;     // [3][tbl_stride] cumulative task counts of the task blocks (n_blocks + 1 used)
+  const int4* blk_info;         // [3][tbl_stride] {0: GEMM-1 / 1: GEMM-2, expert, first row tile, row tiles}
+  const int32_t* n_blocks;      // [3] device scalars
+  int tbl_stride;
+  int part_g1;                  // SM partition: CTAs [0, part_g1) take GEMM-1 tiles, the rest GEMM-2 tiles; 0: none
   int32_t* done;                // tracker: parts stored per 128-row tile of h (zeroed before the launch)
   int E, d, f, n1, n2;          // n1 = ceil(f / 128) GEMM-1 column tiles, n2 = ceil(d / 256) GEMM-2 column tiles
   int32_t* status;

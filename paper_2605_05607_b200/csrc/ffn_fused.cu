@@ -42,14 +42,15 @@ struct Task {
   int mt_global;   // index of the 128-row tile of h among all tiles (tracker slot)
 };
 
-__device__ __forceinline__ Task decode_task(int w, const FusedParams& p, int nb) {
+__device__ __forceinline__ Task decode_task(int w, const FusedParams& p, const int32_t* blk_start,
+                                            const int4* blk_info, int nb) {
   int lo = 0, hi = nb;   // blk_start[lo] <= w < blk_start[hi]
   while (hi - lo > 1) {
     const int mid = (lo + hi) >> 1;
-    if (__ldg(p.blk_start + mid) <= w) lo = mid; else hi = mid;
+    if (__ldg(blk_start + mid) <= w) lo = mid; else hi = mid;
   }
-  const int4 info = __ldg(p.blk_info + lo);   // {type, expert, first row tile, row tiles}
-  const int local = w - __ldg(p.blk_start + lo);
+  const int4 info = __ldg(blk_info + lo);   // {type, expert, first row tile, row tiles}
+  const int local = w - __ldg(blk_start + lo);
   Task t;
   t.type = info.x;
   t.e = info.y;
@@ -113,8 +114,18 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int nb = __ldg(p.n_blocks);
-  const int total = __ldg(p.blk_start + nb);
+  // Task list of this CTA.  Default: every CTA walks the interleaved list (tasks blockIdx, blockIdx + grid, ...).
+  // SM partition (Sec. IV: thread blocks are divided among the stages): the first `p.part_g1` CTAs take only
+  // GEMM-1 tiles, the others only GEMM-2 tiles, each group walking the list of its own kind; the GEMM-2 group is
+  // paced purely by the tracker, the GEMM-1 group never waits.
+  const bool part = p.part_g1 > 0;
+  const int kind = part ? ((int)blockIdx.x < p.part_g1 ? 0 : 1) : 0;
+  const int32_t* tbl_start = part ? p.blk_start + (size_t)(1 + kind) * p.tbl_stride : p.blk_start;
+  const int4* tbl_info = part ? p.blk_info + (size_t)(1 + kind) * p.tbl_stride : p.blk_info;
+  const int nb = __ldg(p.n_blocks + (part ? 1 + kind : 0));
+  const int total = __ldg(tbl_start + nb);
+  const int first = part ? (kind ? (int)blockIdx.x - p.part_g1 : (int)blockIdx.x) : (int)blockIdx.x;
+  const int stride = part ? (kind ? (int)gridDim.x - p.part_g1 : p.part_g1) : (int)gridDim.x;
   const int KB1 = (p.d + BK - 1) / BK, KB2 = (p.f + BK - 1) / BK;
   volatile int* abort_flag = abort_s;
   const volatile int* global_abort = p.status + ST_ABORT;
@@ -128,8 +139,8 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
   if (warp < 4) {
     // ================================ epilogue ================================
     int tl = 0;
-    for (int w = blockIdx.x; w < total && !*abort_flag; w += gridDim.x, ++tl) {
-      const Task t = decode_task(w, p, nb);
+    for (int w = first; w < total && !*abort_flag; w += stride, ++tl) {
+      const Task t = decode_task(w, p, tbl_start, tbl_info, nb);
       const int buf = tl & 1;
       if (!ptx::mbar_wait_warp<true>(tfull_bar(buf), (tl >> 1) & 1, abort_flag, global_abort)) { timeout(1); break; }
       ptx::tc_fence_after();
@@ -225,8 +236,8 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
     // ================================ TMA producer (weights) ================================
     if (lane == 0) {
       uint32_t it = 0;
-      for (int w = blockIdx.x; w < total && !*abort_flag; w += gridDim.x) {
-        const Task t = decode_task(w, p, nb);
+      for (int w = first; w < total && !*abort_flag; w += stride) {
+        const Task t = decode_task(w, p, tbl_start, tbl_info, nb);
         const int KB = t.type ? KB2 : KB1;
         const CUtensorMap* lo_map = t.type ? &map_w2 : &map_w1;
         const CUtensorMap* hi_map = t.type ? &map_w2 : &map_w3;
@@ -255,8 +266,8 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
       const uint64_t b_base = desc_base(BK * 128, 1024);
       uint32_t it = 0;
       int tl = 0;
-      for (int w = blockIdx.x; w < total && !*abort_flag; w += gridDim.x, ++tl) {
-        const Task t = decode_task(w, p, nb);
+      for (int w = first; w < total && !*abort_flag; w += stride, ++tl) {
+        const Task t = decode_task(w, p, tbl_start, tbl_info, nb);
         const int KB = t.type ? KB2 : KB1;
         const int buf = tl & 1;
         if (!ptx::mbar_wait(tempty_bar(buf), ((tl >> 1) & 1) ^ 1, abort_flag, global_abort)) { timeout(3); break; }
@@ -286,8 +297,8 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
     const int chunk = gt & 7;             // 16-byte chunk of the 128-byte K row
     const int rbase = gt >> 3;            // rows rbase + 16 j
     uint32_t it = 0;
-    for (int w = blockIdx.x; w < total && !*abort_flag; w += gridDim.x) {
-      const Task t = decode_task(w, p, nb);
+    for (int w = first; w < total && !*abort_flag; w += stride) {
+      const Task t = decode_task(w, p, tbl_start, tbl_info, nb);
       const int KB = t.type ? KB2 : KB1;
       const int K = t.type ? p.f : p.d;
       const uint8_t* base = static_cast<const uint8_t*>(t.type ? (const void*)p.h : p.x);
@@ -360,38 +371,33 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
   }
 }
 
-// Task blocks in emission order (one thread: at most E + P / 2048 blocks of each kind).
+// Task blocks (one thread: at most E + P / 2048 blocks of each kind).  Three tables, `stride` entries apart:
+// 0: both kinds interleaved in emission order, 1: the GEMM-1 blocks alone, 2: the GEMM-2 blocks alone.
 __global__ void ffn_task_table_kernel(const int32_t* __restrict__ expert_counts, int E, int n1, int n2,
-                                      int32_t* blk_start, int4* blk_info, int32_t* n_blocks) {
+                                      int32_t* blk_start, int4* blk_info, int32_t* n_blocks, int stride) {
   grid_dependency_sync();
   if (threadIdx.x != 0 || blockIdx.x != 0) return;
-  int nb = 0, acc = 0;
+  int nb = 0, acc = 0, nb1 = 0, acc1 = 0, nb2 = 0, acc2 = 0;
+  int32_t *s1 = blk_start + stride, *s2 = blk_start + 2 * stride;
+  int4 *i1 = blk_info + stride, *i2 = blk_info + 2 * stride;
   int pe = -1, pm0 = 0, pmc = 0;   // previous GEMM-1 block, whose GEMM-2 block follows the next GEMM-1 block
+  auto emit2 = [&](int e, int m0, int mc) {
+    blk_start[nb] = acc; blk_info[nb] = make_int4(1, e, m0, mc); acc += mc * n2; ++nb;
+    s2[nb2] = acc2; i2[nb2] = make_int4(1, e, m0, mc); acc2 += mc * n2; ++nb2;
+  };
   for (int e = 0; e < E; ++e) {
     const int M = (expert_counts[e] + BM - 1) / BM;
     for (int m0 = 0; m0 < M; m0 += M_BLOCK) {
       const int mc = min(M_BLOCK, M - m0);
-      blk_start[nb] = acc;
-      blk_info[nb] = make_int4(0, e, m0, mc);
-      acc += mc * n1;
-      ++nb;
-      if (pe >= 0) {
-        blk_start[nb] = acc;
-        blk_info[nb] = make_int4(1, pe, pm0, pmc);
-        acc += pmc * n2;
-        ++nb;
-      }
+      blk_start[nb] = acc; blk_info[nb] = make_int4(0, e, m0, mc); acc += mc * n1; ++nb;
+      s1[nb1] = acc1; i1[nb1] = make_int4(0, e, m0, mc); acc1 += mc * n1; ++nb1;
+      if (pe >= 0) emit2(pe, pm0, pmc);
       pe = e; pm0 = m0; pmc = mc;
     }
   }
-  if (pe >= 0) {
-    blk_start[nb] = acc;
-    blk_info[nb] = make_int4(1, pe, pm0, pmc);
-    acc += pmc * n2;
-    ++nb;
-  }
-  blk_start[nb] = acc;
-  *n_blocks = nb;
+  if (pe >= 0) emit2(pe, pm0, pmc);
+  blk_start[nb] = acc; s1[nb1] = acc1; s2[nb2] = acc2;
+  n_blocks[0] = nb; n_blocks[1] = nb1; n_blocks[2] = nb2;
 }
 
 }  // namespace
@@ -411,7 +417,7 @@ cudaError_t launch_ffn_fused(const FusedParams& p, const int32_t* expert_counts,
   cudaError_t err = cudaMemsetAsync(p.done, 0, done_entries * sizeof(int32_t), st);
   if (err != cudaSuccess) return err;
   if ((err = launch_pdl(ffn_task_table_kernel, 1, 32, 0, st, expert_counts, p.E, p.n1, p.n2, blk_start, blk_info,
-                        n_blocks)) != cudaSuccess)
+                        n_blocks, p.tbl_stride)) != cudaSuccess)
     return err;
   ProfileScope prof(KID_GEMM1, st);
   return launch_pdl(ffn_fused_kernel, sm_count(), THREADS, SMEM_BYTES, st, m_w1, m_w3, m_w2, p);

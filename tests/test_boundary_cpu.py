@@ -70,13 +70,13 @@ def test_bad_shapes_rejected(lib, kw, code):
 
 def test_bad_flags_rejected(lib):
     with pytest.raises(B.MoEError) as ei:
-        B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=16))
+        B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=32))
     assert ei.value.code == B.MOE_ERR_INVALID_ARG
     # the weight cannot be applied in Combine when Combine happens inside GEMM-2's epilogue
     with pytest.raises(B.MoEError) as ei:
         B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=3))
     assert ei.value.code == B.MOE_ERR_INVALID_ARG
-    for ok in (0, 1, 2, 4, 5, 8, 9):
+    for ok in (0, 1, 2, 4, 5, 8, 9, 24):
         assert B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=ok)) > 0
     # k = 1: the fp32 token accumulators are larger than o and the workspace accounts for them
     c = synth.CONFIGS["C1"].with_(k=1)

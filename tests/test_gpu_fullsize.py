@@ -165,10 +165,12 @@ def test_fullsize_single_kernel_ffn_equals_two_kernels(name):
     run.dispatch()
     run.ffn()
     o_two = run.o.clone()
-    fused = H.Run(cfg, B.MOE_FLAG_FUSED_FFN, inputs=run.t)
-    fused.idx, fused.w, fused.lay, fused.xg = run.idx, run.w, run.lay, run.xg
-    fused.o.fill_(3.0)
-    fused.ffn()
-    torch.cuda.synchronize()
-    assert fused.status()[0] == 0
-    assert torch.equal(fused.o[: cfg.P], o_two[: cfg.P])
+    for flags in (B.MOE_FLAG_FUSED_FFN, B.MOE_FLAG_FUSED_FFN | B.MOE_FLAG_SM_PARTITION):
+        fused = H.Run(cfg, flags, inputs=run.t)
+        fused.idx, fused.w, fused.lay, fused.xg = run.idx, run.w, run.lay, run.xg
+        fused.o.fill_(3.0)
+        fused.ffn()
+        torch.cuda.synchronize()
+        assert fused.status()[0] == 0, flags
+        assert torch.equal(fused.o[: cfg.P], o_two[: cfg.P]), flags
+        del fused

@@ -467,7 +467,12 @@ def test_single_kernel_ffn_with_tile_tracker(cfg):
     o_two = run.o.clone()
     run.layer()
     y_two = run.y.clone()
-    fused = H.Run(cfg, B.MOE_FLAG_FUSED_FFN, inputs=run.t)
+    for flags in (B.MOE_FLAG_FUSED_FFN, B.MOE_FLAG_FUSED_FFN | B.MOE_FLAG_SM_PARTITION):
+        _check_single_kernel(cfg, run, flags, o_two, y_two)
+
+
+def _check_single_kernel(cfg, run, flags, o_two, y_two):
+    fused = H.Run(cfg, flags, inputs=run.t)
     fused.route()
     fused.dispatch()
     for _ in range(2):
