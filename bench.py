@@ -352,6 +352,9 @@ def main():
                     help="multi-GPU form: replicas (default: weights replicated, tokens sharded, no data-path "
                          "collective) or ep (expert parallelism: group g on rank g, all-to-all of the dispatched rows "
                          "and of the pre-reduced rows; needs E % N == 0; bf16 experts)")
+    ap.add_argument("--layer-flags", type=int, default=0,
+                    help="MOE_FLAG_* bits for the timed moe_layer call (2: Combine in GEMM-2's epilogue, 8: GEMM-1 + GEMM-2 "
+                         "as one tracker-paced kernel, 24: the same with the SM partition); default 0")
     ap.add_argument("--lean", action="store_true",
                     help="timed region only: no e2e / stage / cpu_baseline legs (for profiler captures)")
     ap.add_argument("--stages-only", action="store_true",
@@ -394,7 +397,7 @@ def main():
     # weights replicated (same seed on every rank), tokens differ per rank
     from paper_2605_05607_b200 import replicas
     t = replicas.make_rank_inputs(cfg, rank, "cuda")
-    shape = B.make_shape(cfg)
+    shape = B.make_shape(cfg, args.layer_flags)
     ws = B.alloc_workspace(shape)
     y = torch.zeros(cfg.T, cfg.d, dtype=torch.bfloat16, device="cuda")
 
@@ -573,6 +576,8 @@ def main():
                          "(geomean 1.59x) on a SIMULATED 32-GPU GH200 NVL32 (BookSim2 + Accel-Sim, H200-configured "
                          "GPUs, NVLink 4, FP8 GEMMs); no tokens/s, GB/s or TFLOP/s for this path, hence vs_baseline null",
     }
+    if args.layer_flags:
+        line["config"]["layer_flags"] = args.layer_flags
     if ep_rank is not None:
         line["config"]["parallelism"] = (f"expert parallel x{world}: {cfg.m} experts per GPU, all-to-all of one row per "
                                          "(token, group) out and one pre-reduced row back; split sizes read back once per layer")
