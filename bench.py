@@ -1,10 +1,12 @@
 """Benchmark of the fused MoE layer (gate -> layout -> expert FFN -> combine) on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C2] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C5a] [--impl reference]
 
-One step = one pass of the whole hot path (moe_layer) over one batch of synthetic tokens.
-N > 1 (launched by torchrun): every rank runs an independent replica on its own tokens (weights
-replicated, tokens sharded, no data-path collective) - weak scaling.  Rank 0 prints ONE JSON line.
+One step = one pass of the whole hot path (moe_layer) over one batch of synthetic tokens; the default
+workload is the largest single-GPU configuration (C5a, the DeepSeek-V3-shaped layer).
+N > 1: every rank runs an independent replica on its own tokens (weights replicated, tokens sharded,
+no data-path collective) - weak scaling.  Under torchrun the ranks are the launcher's; without it
+`--gpus N` starts the N ranks itself.  Rank 0 prints ONE JSON line.
 `--impl reference` times the CPU oracle on a bounded token sample instead (rank 0 only).
 """
 from __future__ import annotations
@@ -30,9 +32,13 @@ METRIC = "fused MoE layer tokens/sec"
 UNIT = "tokens/s"
 KERNELS_PER_STEP = 10  # gate split, gate, topk, masks, scan, offsets, fill, gemm1, gemm2, combine
 
-# DRAM bytes (read + write) of one GEMM-1 launch from ncu captures summarised under profiles/;
-# None until a capture of that workload exists.
-GEMM1_DRAM_TRAFFIC = {"C2": 1.960784e9 + 229.266e6}   # profiles/ffn_gemm_C2_ncu_full.md
+NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16 data-sheet figure, for context beside the measured peaks
+BURST_REGION_S = 1.0           # a timed region shorter than this runs before the power cap settles: burst peak
+CPU_SAMPLE_TOKENS = 16         # tokens per oracle pass, the same for the cpu_baseline leg and the reference arm
+
+# DRAM bytes (read + write) of one GEMM-1 launch, dram__bytes_read.sum + dram__bytes_write.sum of a
+# single-pass ncu capture of that workload; absent: null in the line.
+GEMM1_DRAM_TRAFFIC = {"C2": 1.960784e9 + 229.266e6, "C5a": 21.76e9 + 1.07e9}
 
 
 def peaks():
@@ -59,7 +65,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                                          "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             return
         def pump():
@@ -92,12 +98,23 @@ class ClockSampler:
                 "power_w_max": max(float(f[3]) for f in rows), "reasons": sorted(reasons), "samples": len(rows)}
 
 
+class ExpertSlabs:
+    """Indexable by expert: the raw bf16 bits of that expert's weight matrix on the host.  The oracle
+    takes one expert at a time, so a 22 GB weight set never has to sit in host memory as a whole."""
+
+    def __init__(self, w):
+        self.w = w
+
+    def __getitem__(self, e):
+        return synth.bf16_bits(self.w[int(e)])
+
+
 def oracle_sample_run(cfg, t, sample: int):
     """Time the CPU oracle (as it stands) on `sample` tokens of the workload; returns seconds."""
     from oracle import moe_oracle as O
     bits = synth.bf16_bits
     xb = bits(t["x"])
-    w1, w3, w2 = bits(t["w1"]), bits(t["w3"]), bits(t["w2"])
+    w1, w3, w2 = ExpertSlabs(t["w1"]), ExpertSlabs(t["w3"]), ExpertSlabs(t["w2"])
     wg = t["w_gate"].cpu().numpy()
     bias = None if t["bias"] is None else t["bias"].cpu().numpy()
     toks = synth.sample_tokens(cfg, sample)
@@ -124,12 +141,7 @@ def run_reference(args, cfg):
     if rank != 0:
         return
     t = synth.make_inputs(cfg, "cpu")
-    sample = args.ref_sample
-    if sample <= 0:
-        # size the per-step sample so that the whole run stays within ~200 s: one token is timed
-        # first; n tokens never cost more than n times that (weight decoding is shared)
-        dt1, _ = oracle_sample_run(cfg, t, 1)
-        sample = int(max(1, min(64, 200.0 / (args.steps + args.warmup) / dt1)))
+    sample = args.cpu_sample or CPU_SAMPLE_TOKENS   # the same token sample as the cpu_baseline leg of the GPU arm
     times = []
     for i in range(args.warmup + args.steps):
         dt, n = oracle_sample_run(cfg, t, sample)
@@ -327,24 +339,68 @@ def workload_config(cfg, n_gpus):
                   (6.0 * cfg.E * cfg.d * cfg.f / 1e9)}
 
 
+def self_launch(n: int) -> int:
+    """`python bench.py --gpus N` outside a launcher: start the N ranks under torch.distributed.run (one
+    process per GPU, rendezvous on 127.0.0.1) with the same arguments and return its exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def check_world(args, world: int) -> None:
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s); "
+                         "they must agree (n_gpus in the JSON line is the real world size)")
+
+
+def launcher_selftest(args) -> None:
+    """The launch / barrier / max-over-ranks skeleton of the benchmark with a stub step, on gloo."""
+    from paper_2605_05607_b200 import replicas
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        sys.exit(self_launch(args.gpus))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    check_world(args, world)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("gloo")
+        dist.barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        time.sleep(0.001 * (1 + rank))          # stub step: rank r takes (1 + r) ms
+    ms = replicas.max_over_ranks((time.perf_counter() - t0) * 1e3, dist, "cpu")
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"launcher_selftest": True, "n_gpus": world, "steps": args.steps,
+                          "ms_per_step": ms / args.steps}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None,
-                    help="timed steps (default 200: ~0.5 s on C2, long enough for clock samples; reference arm: 8)")
+                    help="timed steps (default 100: ~2 s on C5a, the sustained regime, with clock samples inside the "
+                         "region; reference arm: 8)")
     ap.add_argument("--warmup", type=int, default=None, help="untimed warm-up steps (default 10; reference arm: 2)")
-    ap.add_argument("--config", default="C2", choices=sorted(synth.ALL_CONFIGS),
+    ap.add_argument("--config", default="C5a", choices=sorted(synth.ALL_CONFIGS),
                     help="C1..C5b: the benchmark configurations; S8..L32: the paper's Small/Medium/Large shapes "
                          "at top-k 8/16/32 (Table 'Model Configurations')")
     ap.add_argument("--paper-shapes", action="store_true",
                     help="with --report: also run the nine Small/Medium/Large x top-k shapes")
     ap.add_argument("--shape", default=None, metavar="T,d,f,E,k,G",
-                    help="override the sizes of --config (keeps its score function and router bias); "
-                         "for profiler captures of a slice that fits the capture size rules")
+                    help="override the sizes of --config (keeps its score function and router bias), e.g. a "
+                         "slice of a large layer with the same per-expert geometry for a profiler capture")
     ap.add_argument("--impl", default="tcmoe", choices=["tcmoe", "reference"])
-    ap.add_argument("--ref-sample", type=int, default=0,
-                    help="tokens per step of the reference arm (0: sized from a one-token calibration)")
-    ap.add_argument("--cpu-sample", type=int, default=1024, help="tokens of the cpu_baseline leg (0: skip)")
+    ap.add_argument("--cpu-sample", type=int, default=CPU_SAMPLE_TOKENS,
+                    help="tokens per CPU-oracle pass: the cpu_baseline leg (0: skip it) and every step of the "
+                         "reference arm use the same sample")
     ap.add_argument("--experts", default="bf16", choices=["bf16", "fp8"],
                     help="bf16 (the benchmark's precision, default) or fp8: E4M3 experts through moe_layer_fp8 "
                          "(per-token / per-output-column scales; gate and combine stay bf16 / fp32)")
@@ -355,6 +411,9 @@ def main():
     ap.add_argument("--layer-flags", type=int, default=0,
                     help="MOE_FLAG_* bits for the timed moe_layer call (2: Combine in GEMM-2's epilogue, 8: GEMM-1 + GEMM-2 "
                          "as one tracker-paced kernel, 24: the same with the SM partition); default 0")
+    ap.add_argument("--launcher-selftest", action="store_true",
+                    help="exercise the multi-rank launcher and the max-over-ranks timing with a stub step on the "
+                         "gloo backend (no GPU, no library); prints the JSON line's n_gpus / steps / ms_per_step")
     ap.add_argument("--lean", action="store_true",
                     help="timed region only: no e2e / stage / cpu_baseline legs (for profiler captures)")
     ap.add_argument("--stages-only", action="store_true",
@@ -365,7 +424,7 @@ def main():
                     help="also write per-stage numbers of every configuration to this JSON file (1 GPU)")
     args = ap.parse_args()
     if args.steps is None:
-        args.steps = 200 if args.impl == "tcmoe" else 8
+        args.steps = 100 if args.impl == "tcmoe" else 8
     if args.warmup is None:
         args.warmup = 10 if args.impl == "tcmoe" else 2
     args.warmup = max(args.warmup, 3) if args.impl == "tcmoe" else args.warmup
@@ -378,6 +437,12 @@ def main():
         run_reference(args, cfg)
         return
 
+    if args.launcher_selftest:
+        launcher_selftest(args)
+        return
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        sys.exit(self_launch(args.gpus))
+
     from paper_2605_05607_b200 import binding as B
     B.lib()  # fail loudly if the CUDA library is missing
     if args.stages_only:
@@ -388,10 +453,13 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    check_world(args, world)
     torch.cuda.set_device(local)
     dist = None
     if world > 1:
         import torch.distributed as dist
+        os.environ.setdefault("NCCL_DEBUG", "INFO")       # the communicator lines show the rank count
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     # weights replicated (same seed on every rank), tokens differ per rank
@@ -546,10 +614,16 @@ def main():
     pk = peaks()
     tokens = cfg.T * world * args.steps
     value = replicas.whole_job_tokens_per_s(cfg, world, args.steps, elapsed_ms)
-    flops_g1 = 4.0 * cfg.P * cfg.d * cfg.f                      # GEMM-1: x W1 and x W3
+    flops_g1 = 4.0 * cfg.P * cfg.d * cfg.f                      # GEMM-1: x W1 and x W3, useful rows only
     g1_avg_s = (g1_ms / max(g1_launches, 1)) * 1e-3
     achieved = flops_g1 / g1_avg_s / 1e12 if g1_launches else None
-    peak = pk["bf16_tflops_sustained"] * (2.0 if fp8 else 1.0)
+    # Denominator by the length of the timed region: a region of well under a second after an idle GPU runs
+    # at boost clocks (the burst peak applies); a longer one sits at the power cap (the sustained peak).
+    scale = 2.0 if fp8 else 1.0                                  # nominal fp8 : bf16 ratio; no measured fp8 peak
+    region_s = elapsed_ms * 1e-3
+    burst = region_s < BURST_REGION_S
+    peak = (pk["bf16_tflops"] if burst else pk["bf16_tflops_sustained"]) * scale
+    frac_of = (lambda denom: (achieved / (denom * scale)) if achieved else None)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": elapsed_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -567,8 +641,13 @@ def main():
         "roofline": {"kernel": "ffn_gemm1_kernel (GEMM-1 + SwiGLU, tcgen05)", "bound": "tensor",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": (achieved / peak) if achieved else None,
-                     "peak_source": f"{pk['source']} bf16 sustained (kernel timed inside a long step)" +
-                                    (" x 2 (nominal fp8 : bf16 ratio; no measured fp8 peak)" if fp8 else ""),
+                     "frac_burst": frac_of(pk["bf16_tflops"]), "frac_sustained": frac_of(pk["bf16_tflops_sustained"]),
+                     "frac_nominal": frac_of(NOMINAL_BF16_TFLOPS),
+                     "peak_source": (f"{pk['source']} bf16 " + ("burst" if burst else "sustained") +
+                                     f" (timed region {region_s:.2f} s, burst below {BURST_REGION_S:.0f} s)" +
+                                     (" x 2 (nominal fp8 : bf16 ratio; no measured fp8 peak)" if fp8 else "")),
+                     "peaks": {"burst": pk["bf16_tflops"] * scale, "sustained": pk["bf16_tflops_sustained"] * scale,
+                               "nominal": NOMINAL_BF16_TFLOPS * scale},
                      "flops_per_launch": flops_g1, "avg_launch_ms": g1_avg_s * 1e3, "launches": g1_launches,
                      "traffic": None if fp8 else GEMM1_DRAM_TRAFFIC.get(cfg.name)},
         "ffn_tflops_layer": 6.0 * cfg.P * cfg.d * cfg.f * args.steps / (elapsed_ms * 1e-3) / 1e12,
@@ -588,6 +667,19 @@ def main():
         del wq, sc
     if world == 1 and not args.lean and ep_rank is None:
         line["stages"] = stage_breakdown(cfg, t)
+        st = line["stages"]
+        # the two memory-bound kernels the metric names, isolated (cold L2) and, for combine, right behind the GEMMs
+        line["hbm_kernels"] = {
+            "peak": pk["hbm_gbs"], "unit": "GB/s", "peak_source": f"{pk['source']} copy bandwidth",
+            "dispatch": {"achieved": st["dispatch"]["gbs"], "frac": st["dispatch"]["frac_hbm_measured"],
+                         "bytes": st["dispatch"]["bytes"]},
+            "combine": {"achieved": st["combine"]["gbs"], "frac": st["combine"]["frac_hbm_measured"],
+                        "bytes": st["combine"]["bytes"], "achieved_in_layer": st["combine"]["in_layer_gbs"],
+                        "frac_in_layer": st["combine"]["in_layer_gbs"] / pk["hbm_gbs"]}}
+        line["ffn_tflops_isolated"] = {k: st["expert_ffn"][k] for k in ("tflops", "gemm1_tflops", "gemm2_tflops",
+                                                                          "frac_bf16_burst", "frac_bf16_sustained")}
+        line["fused_vs_unfused_ms"] = {k: st["summary"][k] for k in ("fused_back_to_back_ms", "unfused_back_to_back_ms",
+                                                                      "fused_ms", "unfused_sum_ms")}
     if world == 1 and args.report and not args.lean:
         report = {cfg.name: line["stages"]}
         del t

@@ -61,7 +61,7 @@ enum { MOE_SCORE_SOFTMAX = 0,      /* weights = softmax over the k selected keys
 enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1,   /* default (0): gate weight applied in GEMM-2's
                                             epilogue, Combine un-weighted (Sec. III-C)    */
        MOE_FLAG_COMBINE_IN_EPILOGUE = 2, /* moe_layer only: Combine runs inside GEMM-2's
-                                            epilogue (Sec. V, fused pipeline): every weighted
+                                            epilogue (Sec. IV, fused pipeline): every weighted
                                             expert row is added into an fp32 accumulator row of
                                             its token with vector reductions, o is never
                                             written, a last pass rounds the accumulators to
@@ -85,6 +85,11 @@ enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1,   /* default (0): gate weight applied in 
                                             SMs take only GEMM-1 tiles, one third only GEMM-2
                                             tiles, the second group paced by the tracker alone.
                                             Same results.                                      */
+       MOE_FLAG_GEMM2_PAIR = 32,         /* GEMM-2 runs on 256-row CTA-pair tiles (cta_group::2) whatever the shape */
+       MOE_FLAG_GEMM2_SINGLE = 64,       /* GEMM-2 runs on 128-row single-CTA tiles whatever the shape.  Without either
+                                            flag the library picks from the shape: pair tiles unless experts hold
+                                            fewer than 512 rows on average.  The two flags exclude each other; the
+                                            results of both forms meet the same tolerances.               */
        MOE_FLAG_FUSED_FFN = 8 };         /* moe_expert_ffn / moe_layer (bf16 experts): GEMM-1 and
                                             GEMM-2 run as ONE persistent kernel paced by a tile
                                             tracker (Sec. IV token-centric kernel fusion, tiles of
@@ -194,7 +199,7 @@ int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, co
                    void* ws, size_t ws_bytes, void* stream);
 
 /* ---- FP8 form of the expert FFN --------------------------------------------------------------
- * Sec. VI-A evaluates the DeepSeek-V3 experts with FP8 GEMM kernels and gives no recipe; this
+ * Sec. V-A evaluates the DeepSeek-V3 experts with FP8 GEMM kernels and gives no recipe; this
  * library's reading: E4M3 elements (largest finite value 448, round to nearest even, saturating),
  * one fp32 scale per activation row and one per (expert, output column) of a weight matrix,
  * scale = fl32(max|v| / 448) (1 for an all-zero vector), code = e4m3(fl32(v / scale)); fp32
@@ -249,8 +254,12 @@ int moe_layer_fp8_host(const moe_shape_t* shape, const void* x_host, void* x_dev
  *    dispatched copy), bit for bit.  The call allocates nothing and frees nothing.
  *  - Limit: 256 + 8*(E+G)*ceil(T/32) + 8*(E+1) bytes (each table rounded up to 256) must fit in
  *    MOE_NOALLOC_SCRATCH_BYTES; larger shapes return MOE_ERR_SCRATCH_LIMIT and launch nothing.
- *  - The first call on a device looks up the array's device address; make that first call
- *    outside any stream capture.  Later calls only enqueue work on `stream`.
+ *  - The array used is the CURRENT device's copy (cudaGetDevice at the time of the call): `stream`
+ *    and every pointer must belong to that device.
+ *  - The first call on a device looks up the array's device address, which also makes the CUDA
+ *    runtime load the library's device code there (an implicit allocation and synchronisation by
+ *    the runtime, once); make that first call outside any stream capture.  "Allocates nothing"
+ *    holds for every later call, which only enqueues work on `stream`.
  *  - All calls on a device share the array and it keeps the previous call's contents; the
  *    entry point clears what must start at zero.  Two calls that overlap on the GPU (different
  *    streams, no ordering between them) race on it: serialise them.
@@ -269,8 +278,8 @@ int moe_workspace_layout(const moe_shape_t* shape, size_t out[4]);
 enum { MOE_KERNEL_TOPK = 1, MOE_KERNEL_MASKS = 2, MOE_KERNEL_FILL = 3, MOE_KERNEL_DISPATCH = 4,
        MOE_KERNEL_GEMM1 = 5, MOE_KERNEL_GEMM2 = 6, MOE_KERNEL_COMBINE = 7, MOE_KERNEL_GATE = 8 };
 
-/* Per-kernel timing hook for benchmarks (host-side state, one per process; not part of the
- * method).  After moe_profile_enable(id) every launch of that kernel by any entry point is
+/* Per-kernel timing hook for benchmarks (host-side state, one record per process, guarded by a
+ * mutex so that launches from several host threads are safe; not part of the method).  After moe_profile_enable(id) every launch of that kernel by any entry point is
  * bracketed by a pair of CUDA events on the launching stream (up to 4096 launches; later ones
  * are not recorded).  moe_profile_read waits for the recorded events, returns the summed
  * device time in milliseconds and the number of launches, and clears the record.

@@ -4,7 +4,7 @@ THIS IS TEST INFRASTRUCTURE, NOT PRODUCT CODE.  Only the test-suite and the
 benchmark's baseline legs may import it.  Plain numpy, one step per function,
 no blocking or reordering; it shares no code or table with the CUDA path.
 
-What the paper fixes: Sec. VI-A says only that the DeepSeek-V3 experts are
+What the paper fixes: Sec. V-A says only that the DeepSeek-V3 experts are
 simulated with "FP8 kernels".  Format and scaling are therefore a reading,
 the same on both sides:
 

@@ -35,6 +35,8 @@ MOE_FLAG_COMBINE_IN_EPILOGUE = 2
 MOE_FLAG_SPARSE_TOPK = 4
 MOE_FLAG_FUSED_FFN = 8
 MOE_FLAG_SM_PARTITION = 16
+MOE_FLAG_GEMM2_PAIR = 32
+MOE_FLAG_GEMM2_SINGLE = 64
 
 EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "moe_status", "moe_strerror",
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",

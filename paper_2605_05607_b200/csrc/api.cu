@@ -7,6 +7,9 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+#include <mutex>
+
 namespace tcmoe {
 namespace {
 
@@ -79,8 +82,9 @@ int check_shape(const moe_shape_t* s) {
   if (s->T < 0 || s->d <= 0 || s->f <= 0 || s->E <= 0 || s->k <= 0 || s->G <= 0) return MOE_ERR_INVALID_ARG;
   if (s->score_fn != MOE_SCORE_SOFTMAX && s->score_fn != MOE_SCORE_SIGMOID) return MOE_ERR_INVALID_ARG;
   if (s->flags & ~(MOE_FLAG_WEIGHT_IN_COMBINE | MOE_FLAG_COMBINE_IN_EPILOGUE | MOE_FLAG_SPARSE_TOPK | MOE_FLAG_FUSED_FFN |
-                   MOE_FLAG_SM_PARTITION))
+                   MOE_FLAG_SM_PARTITION | MOE_FLAG_GEMM2_PAIR | MOE_FLAG_GEMM2_SINGLE))
     return MOE_ERR_INVALID_ARG;
+  if ((s->flags & MOE_FLAG_GEMM2_PAIR) && (s->flags & MOE_FLAG_GEMM2_SINGLE)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_SM_PARTITION) && !(s->flags & MOE_FLAG_FUSED_FFN)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_FUSED_FFN) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_WEIGHT_IN_COMBINE) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
@@ -150,15 +154,20 @@ bool have_device() {
 
 namespace tcmoe {
 namespace {
+// State of the timing hook.  One record per process, guarded by a mutex: launches from several host threads
+// may be bracketed while another thread enables, disables or reads the hook.
 constexpr int PROFILE_CAP = 4096;
-int g_profile_id = 0;
+std::mutex g_profile_mutex;
+std::atomic<int> g_profile_id{0};   // read without the lock on the launch path when the hook is off
 int g_profile_n = 0;
 cudaEvent_t g_ev0[PROFILE_CAP], g_ev1[PROFILE_CAP];
 int g_events_made = 0;
 }  // namespace
 
 ProfileScope::ProfileScope(int kernel_id, cudaStream_t s) : slot(-1), st(s) {
-  if (g_profile_id == 0 || kernel_id != g_profile_id || g_profile_n >= PROFILE_CAP) return;
+  if (g_profile_id.load(std::memory_order_relaxed) != kernel_id || kernel_id == 0) return;
+  std::lock_guard<std::mutex> lock(g_profile_mutex);
+  if (g_profile_id.load(std::memory_order_relaxed) != kernel_id || g_profile_n >= PROFILE_CAP) return;
   while (g_events_made <= g_profile_n) {
     if (cudaEventCreate(&g_ev0[g_events_made]) != cudaSuccess || cudaEventCreate(&g_ev1[g_events_made]) != cudaSuccess)
       return;
@@ -168,7 +177,9 @@ ProfileScope::ProfileScope(int kernel_id, cudaStream_t s) : slot(-1), st(s) {
   cudaEventRecord(g_ev0[slot], st);
 }
 ProfileScope::~ProfileScope() {
-  if (slot >= 0) cudaEventRecord(g_ev1[slot], st);
+  if (slot < 0) return;
+  std::lock_guard<std::mutex> lock(g_profile_mutex);
+  cudaEventRecord(g_ev1[slot], st);
 }
 }  // namespace tcmoe
 
@@ -263,13 +274,15 @@ int moe_selftest_wait_timeout(void* ws, uint64_t limit_ns, void* stream) {
 
 int moe_profile_enable(int kernel_id) {
   if (kernel_id < 0 || kernel_id > 8) return MOE_ERR_INVALID_ARG;
-  g_profile_id = kernel_id;
+  std::lock_guard<std::mutex> lock(g_profile_mutex);
+  g_profile_id.store(kernel_id, std::memory_order_relaxed);
   g_profile_n = 0;
   return MOE_OK;
 }
 
 int moe_profile_read(float* total_ms, int32_t* launches) {
   if (total_ms == nullptr || launches == nullptr) return MOE_ERR_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_profile_mutex);
   float sum = 0.f;
   for (int i = 0; i < g_profile_n; ++i) {
     float ms = 0.f;
@@ -393,6 +406,7 @@ int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t*
   if (!have_device()) return MOE_ERR_CUDA;
   FfnArgs a{};
   a.a_src = xg;
+  a.a_rows = shape->T * (shape->k < shape->G ? shape->k : shape->G);   // capacity of the dispatched buffer
   a.gather_idx = layout->row_src;
   a.gather_div = 1;
   a.w1 = w1;
@@ -459,6 +473,7 @@ int moe_expert_ffn_fp8(const moe_shape_t* shape, const void* xq, const float* sx
   if (!have_device()) return MOE_ERR_CUDA;
   FfnArgs a{};
   a.a_src = xq;
+  a.a_rows = shape->T * (shape->k < shape->G ? shape->k : shape->G);   // capacity of the dispatched buffer
   a.gather_idx = layout->row_src;
   a.gather_div = 1;
   a.w1 = w1q;
@@ -499,7 +514,7 @@ int moe_combine(const moe_shape_t* shape, const void* o, const moe_layout_t* lay
   if ((rc = check_ws(shape, ws, ws_bytes, &p)) != MOE_OK) return rc;
   if (!have_device()) return MOE_ERR_CUDA;
   TCMOE_CUDA(launch_combine(to_shape(*shape), o, to_layout(*layout), topk_idx, topk_w, pg, y,
-                            static_cast<cudaStream_t>(stream)));
+                            at<int32_t>(ws, p.status), static_cast<cudaStream_t>(stream)));
   return MOE_OK;
 }
 
@@ -563,6 +578,7 @@ static int layer_impl(const moe_shape_t* shape, const void* x, const float* w_ga
     a.a_src = at<void>(ws, p.xq);
     TCMOE_CUDA(launch_quantize_rows(x, s.T, s.d, at<void>(ws, p.xq), at<float>(ws, p.sx), st));
   }
+  a.a_rows = s.T;
   a.gather_idx = L.row_pair;   // token of expert row r = row_pair[r] / k
   a.gather_div = s.k;
   a.w1 = w1;
@@ -590,7 +606,7 @@ static int layer_impl(const moe_shape_t* shape, const void* x, const float* w_ga
     return MOE_OK;
   }
   TCMOE_CUDA(fp8 != nullptr ? launch_expert_ffn_fp8(s, a, q, st) : launch_expert_ffn(s, a, st));
-  TCMOE_CUDA(launch_combine(s, a.o, L, idx, tw, nullptr, y, st));
+  TCMOE_CUDA(launch_combine(s, a.o, L, idx, tw, nullptr, y, status, st));
   return MOE_OK;
 }
 

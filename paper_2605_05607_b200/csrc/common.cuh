@@ -86,10 +86,11 @@ cudaError_t launch_tile_prefix(const Shape& s, const int32_t* expert_counts, int
 cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void* xg, cudaStream_t st);
 cudaError_t launch_round_rows(const Shape& s, const float* acc, void* y, cudaStream_t st);
 cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
-                           const float* topk_w, void* pg, void* y, cudaStream_t st);
+                           const float* topk_w, void* pg, void* y, int32_t* status, cudaStream_t st);
 // ffn.cu
 struct FfnArgs {
   const void* a_src;          // GEMM-1 activations: xg (gather_div = 1) or x (gather_div = k)
+  int a_rows;                 // rows of a_src (gather indices are checked against it)
   const int32_t* gather_idx;  // row_src, or row_pair (token = row_pair / k)
   int gather_div;
   const void *w1, *w3, *w2;

@@ -1,5 +1,5 @@
-// Expert-parallel execution of the layer across GPUs (paper Sec. II-A: "Dispatch sends each token to the
-// GPUs hosting its experts, Combine brings the outputs back"; Sec. III-D: one replica per destination, trimmed
+// Expert-parallel execution of the layer across GPUs (paper Sec. II-A: Dispatch sends each token to the
+// GPUs hosting its experts, Combine brings the outputs back; Sec. III-D: one replica per destination, trimmed
 // to that destination's targets; reduction of the outputs of one destination before they travel back).
 // With the G expert groups placed on G GPUs, the data that crosses the links is exactly what the single-GPU
 // path already builds: the dispatched buffer xg (one row per distinct (token, group)) on the way out, one

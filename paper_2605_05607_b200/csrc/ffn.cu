@@ -2,8 +2,6 @@
 // (GEMM-1 + SwiGLU in ffn_gemm1.cu, GEMM-2 + gate weight in ffn_gemm2.cu).
 #include "ffn_common.cuh"
 
-#include <cstdlib>
-
 #include <atomic>
 
 namespace tcmoe {
@@ -104,11 +102,11 @@ int sm_count() {
 
 // Experts holding few rows on average: 256-row CTA-pair tiles would be mostly padding (a Zipf-routed
 // 128-expert layer has most experts below 128 rows), so GEMM-2 takes 128-row single-CTA tiles.  Decided from the
-// shape alone (the routing-dependent counts never visit the host); TCMOE_GEMM2=pair|single overrides for experiments.
+// shape alone (the routing-dependent counts never visit the host); flag bits 32 (MOE_FLAG_GEMM2_PAIR) and 64
+// (MOE_FLAG_GEMM2_SINGLE) force one form.
 static bool small_experts(const Shape& s) {
-  const char* env = getenv("TCMOE_GEMM2");
-  if (env != nullptr && env[0] == 'p') return false;
-  if (env != nullptr && env[0] == 's') return true;
+  if (s.flags & 32) return false;
+  if (s.flags & 64) return true;
   return (long long)s.T * s.k < 512ll * s.E;
 }
 
@@ -123,6 +121,7 @@ static cudaError_t launch_expert_ffn_fused(const Shape& s, const FfnArgs& a, cud
   ffn::FusedParams p{};
   p.x = a.a_src;
   p.x_ld = s.d;
+  p.x_rows = a.a_rows;
   p.gather_idx = a.gather_idx;
   p.gather_div = a.gather_div;
   p.h = static_cast<__nv_bfloat16*>(a.h);
@@ -161,6 +160,7 @@ cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st)
   ffn::GemmParams g1{};
   g1.a_src = static_cast<const __nv_bfloat16*>(a.a_src);
   g1.a_ld = s.d;
+  g1.a_rows = a.a_rows;
   g1.gather_idx = a.gather_idx;
   g1.gather_div = a.gather_div;
   g1.out = static_cast<__nv_bfloat16*>(a.h);
@@ -210,6 +210,7 @@ cudaError_t launch_expert_ffn_fp8(const Shape& s, const FfnArgs& a, const Fp8Arg
   ffn::GemmParams g1{};
   g1.a_src = a.a_src;
   g1.a_ld = s.d;
+  g1.a_rows = a.a_rows;
   g1.gather_idx = a.gather_idx;
   g1.gather_div = a.gather_div;
   g1.out = static_cast<__nv_bfloat16*>(a.h);

@@ -10,7 +10,7 @@
 namespace tcmoe {
 namespace ffn {
 
-constexpr int BM = 128;       // rows per CTA tile (the paper's tsize: 128-token tiles, Sec. VI-H)
+constexpr int BM = 128;       // rows per CTA tile (the paper's tsize: 128-token tiles, Sec. VII-C)
 constexpr int BK = 64;        // K per pipeline stage = one 128-byte swizzle row of bf16
 constexpr int UMMA_N = 256;   // accumulator columns per tile
 constexpr int MAX_E = 1024;
@@ -18,6 +18,7 @@ constexpr int MAX_E = 1024;
 struct GemmParams {
   const void* a_src;            // GEMM-1 gather source (xg or x): bf16, or E4M3 codes in the FP8 form
   int a_ld;                     // elements per source row
+  int a_rows;                   // rows of the gather source: indices outside [0, a_rows) are reported, not read
   const int32_t* gather_idx;    // row_src, or row_pair with gather_div = k (token = row_pair / k)
   int gather_div;
   __nv_bfloat16* out;
@@ -107,6 +108,7 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
 struct FusedParams {
   const void* x;                // GEMM-1 gather source (xg or x), bf16
   int x_ld;
+  int x_rows;                   // rows of x: gather indices outside [0, x_rows) are reported, not read
   const int32_t* gather_idx;
   int gather_div;
   __nv_bfloat16* h;             // [P, f] intermediate

@@ -1,7 +1,7 @@
 // Expert FFN as ONE persistent kernel paced by a tile tracker (paper Sec. IV "token-centric kernel fusion":
 // tiles of 128 tokens move through the stages of the layer as soon as the stage before has produced them;
 // Sec. IV-B/C: tracker tables record which tiles are complete, persistent thread blocks poll them, with a
-// synchronisation tile size of 128 tokens, Sec. VI-H).
+// synchronisation tile size of 128 tokens, Sec. VII-C).
 //
 // Tasks are GEMM-1 tiles (128 rows x 128 columns of h: gathered A, W1 | W3, SwiGLU epilogue) and GEMM-2 tiles
 // (128 rows x 256 columns of o: A = rows of h, W2, gate weight in the epilogue), both on the single-CTA UMMA
@@ -332,6 +332,10 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
           if (t.type == 0) {
             idx = __ldg(p.gather_idx + idx);
             if (p.gather_div > 1) idx /= p.gather_div;
+            if (idx < 0 || idx >= p.x_rows) {   // a table entry that is no row of the source: zero-filled
+              report_error(p.status, DEV_INDEX_OUT_OF_RANGE, KID_GEMM1, t.row0 + lr, idx);
+              continue;
+            }
           }
           src[j] = base + (size_t)idx * ld_bytes;
           live |= 1u << j;

@@ -213,7 +213,7 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
         if (lrow < t.rows) {
           int idx = __ldg(p.gather_idx + t.row0 + lrow);
           if (p.gather_div > 1) idx /= p.gather_div;
-          sa = __ldg(p.a_scale + idx);
+          sa = (idx >= 0 && idx < p.a_rows) ? __ldg(p.a_scale + idx) : 0.f;
         }
         const size_t g = (size_t)t.e * p.N + t.n0;
 #pragma unroll
@@ -354,6 +354,10 @@ ffn_gemm1_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
           if (!PLAIN) {
             idx = __ldg(p.gather_idx + idx);
             if (p.gather_div > 1) idx /= p.gather_div;
+            if (idx < 0 || idx >= p.a_rows) {   // a table entry that is no row of the source: zero-filled
+              report_error(p.status, DEV_INDEX_OUT_OF_RANGE, KID_GEMM1, t.row0 + lr, idx);
+              continue;
+            }
           }
           src[j] = base + (size_t)idx * p.a_ld * ELEM;
           live |= 1u << j;

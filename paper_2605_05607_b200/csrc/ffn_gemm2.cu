@@ -43,7 +43,7 @@ constexpr uint32_t IDESC_F8 = idesc_e4m3(2 * BM);
 constexpr uint32_t HINT = 4000;   // try_wait suspend-time hint (ns), see ptx::mbar_try_wait
 
 // RED = false: rows go to o (bf16), Combine is a later pass.  RED = true: Combine happens here
-// (Sec. V: the fused pipeline reduces expert outputs as GEMM-2 produces them): each weighted row is
+// (Sec. IV: the fused pipeline reduces expert outputs as GEMM-2 produces them): each weighted row is
 // added into the fp32 accumulator row of its token with vector reductions; o is never written.
 // FP8 = true: h rows and weights are E4M3 codes, a stage holds 128 elements of K (the same 128 bytes
 // per row), W2 comes K-major from [E, N, K] as one 128-row box per CTA, and the epilogue applies

@@ -262,8 +262,9 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
                                                       const float* __restrict__ topk_w,
                                                       const int32_t* __restrict__ pair_row,
                                                       const int32_t* __restrict__ al,
-                                                      const int32_t* __restrict__ group_offsets, int T, int k, int m,
-                                                      int vec_per_row, int weighted) {
+                                                      const int32_t* __restrict__ group_offsets, int T, int E, int k,
+                                                      int m, int vec_per_row, int weighted, int n_rows,
+                                                      int32_t* status) {
   grid_dependency_sync();
   __shared__ int s_row[8][32];   // per warp: expert-sorted row of the slot at sorted position p
   __shared__ int s_dst[8][32];   // dispatched row (t, g) of that slot's group
@@ -276,11 +277,22 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
     float my_w = 1.f;
     if (lane < k) {
       const int e = __ldg(topk_idx + (size_t)t * k + lane);
-      if (e >= 0) {   // e < 0: unused slot of a sparse top-k table, sorts behind every real slot and is not read
-        my_g = e / m;
-        my_row = __ldg(pair_row + (size_t)t * k + lane);
-        my_dst = __ldg(group_offsets + my_g) + __ldg(al + (size_t)my_g * T + t);
-        if (weighted) my_w = __ldg(topk_w + (size_t)t * k + lane);
+      // e < 0: unused slot of a sparse top-k table, sorts behind every real slot and is not read.  An expert
+      // index or a row outside its table (the layout builder reported it and wrote row -1) is skipped the
+      // same way, so no table entry is ever used as an address unchecked.
+      if (e >= 0 && e < E) {
+        const int r = __ldg(pair_row + (size_t)t * k + lane);
+        const int a = __ldg(al + (size_t)(e / m) * T + t);
+        if (r >= 0 && r < n_rows && a >= 0) {
+          my_g = e / m;
+          my_row = r;
+          my_dst = __ldg(group_offsets + my_g) + a;
+          if (weighted) my_w = __ldg(topk_w + (size_t)t * k + lane);
+        } else {
+          report_error(status, DEV_INDEX_OUT_OF_RANGE, KID_COMBINE, t, r);
+        }
+      } else if (e >= E) {
+        report_error(status, DEV_INDEX_OUT_OF_RANGE, KID_COMBINE, t, e);
       }
     }
     const int kv = __popc(__ballot_sync(0xFFFFFFFFu, lane < k && my_g != 0x7FFFFFFF));   // slots in use
@@ -325,15 +337,15 @@ __global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ 
 }
 
 cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
-                           const float* topk_w, void* pg, void* y, cudaStream_t st) {
+                           const float* topk_w, void* pg, void* y, int32_t* status, cudaStream_t st) {
   if (s.T == 0) return cudaSuccess;
   int blocks = (s.T + 7) / 8;
   const int cap = sm_count() * 8;
   if (blocks > cap) blocks = cap;
   ProfileScope prof(KID_COMBINE, st);
   return launch_pdl(combine_kernel, blocks, 256, 0, st, static_cast<const uint4*>(o), static_cast<uint4*>(y),
-                    static_cast<uint4*>(pg), topk_idx, topk_w, L.pair_row, L.al, L.group_offsets, s.T, s.k, s.E / s.G,
-                    s.d / 8, (s.flags & 1) ? 1 : 0);
+                    static_cast<uint4*>(pg), topk_idx, topk_w, L.pair_row, L.al, L.group_offsets, s.T, s.E, s.k,
+                    s.E / s.G, s.d / 8, (s.flags & 1) ? 1 : 0, s.T * s.k, status);
 }
 
 // Last step of the layer when Combine ran inside GEMM-2's epilogue: the fp32 token accumulators

@@ -81,11 +81,6 @@ extern "C" int moe_dispatch_noalloc(const moe_shape_t* shape, const void* x, con
   const size_t need = up256(off_mp + (E + 1) * 4);
   if (need > kScratchBytes) return MOE_ERR_SCRATCH_LIMIT;
 
-  int ndev = 0;
-  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev <= 0) {
-    (void)cudaGetLastError();
-    return MOE_ERR_CUDA;
-  }
   void* base = nullptr;
   if ((rc = scratch_of_current_device(&base)) != MOE_OK) return rc;
   unsigned char* b = static_cast<unsigned char*>(base);

@@ -1,4 +1,4 @@
-// bf16 -> E4M3 quantisation for the FP8 form of the expert FFN (paper Sec. VI-A: the evaluated
+// bf16 -> E4M3 quantisation for the FP8 form of the expert FFN (paper Sec. V-A: the evaluated
 // DeepSeek-V3 experts run FP8 GEMMs; format and scaling are this library's reading):
 //   scale = fl32(max|v| / 448) over a row (activations) or over K for one (expert, output column)
 //           (weights); 1 for an all-zero vector
@@ -64,6 +64,7 @@ __global__ void __launch_bounds__(256) quantize_weights_kernel(const __nv_bfloat
   __shared__ float red[8][32];
   __shared__ float sc_s[32];
   __shared__ uint8_t tile[32][33];
+  grid_dependency_sync();
   const int e = blockIdx.y, n0 = blockIdx.x * 32;
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;   // tx: column (pass 1 / tile load), ty: 0..7
   const __nv_bfloat16* we = w + (size_t)e * K * N;

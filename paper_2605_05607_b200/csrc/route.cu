@@ -1,4 +1,4 @@
-// Routing of the MoE layer (paper Sec. II-A: "topk experts selected by the gate network"); the
+// Routing of the MoE layer (paper Sec. II-A: the gate network selects topk experts per token); the
 // gate logits themselves are computed in gate_gemm.cu.
 //   topk_kernel : key = logit + bias; k largest keys per token ordered by
 //                 (key descending, expert index ascending); gate weights over the k keys

@@ -70,13 +70,16 @@ def test_bad_shapes_rejected(lib, kw, code):
 
 def test_bad_flags_rejected(lib):
     with pytest.raises(B.MoEError) as ei:
-        B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=32))
+        B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=1 << 12))
+    assert ei.value.code == B.MOE_ERR_INVALID_ARG
+    with pytest.raises(B.MoEError) as ei:   # the two forced GEMM-2 forms exclude each other
+        B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=B.MOE_FLAG_GEMM2_PAIR | B.MOE_FLAG_GEMM2_SINGLE))
     assert ei.value.code == B.MOE_ERR_INVALID_ARG
     # the weight cannot be applied in Combine when Combine happens inside GEMM-2's epilogue
     with pytest.raises(B.MoEError) as ei:
         B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=3))
     assert ei.value.code == B.MOE_ERR_INVALID_ARG
-    for ok in (0, 1, 2, 4, 5, 8, 9, 24):
+    for ok in (0, 1, 2, 4, 5, 8, 9, 24, 32, 64):
         assert B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=ok)) > 0
     # k = 1: the fp32 token accumulators are larger than o and the workspace accounts for them
     c = synth.CONFIGS["C1"].with_(k=1)
@@ -127,6 +130,32 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(B, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no CPU fallback"):
         B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"]))
+
+
+def test_every_kernel_waits_for_its_stream_predecessor():
+    """All kernels are launched with programmatic stream serialisation, so each must call
+    grid_dependency_sync() before it touches global memory: a kernel without it could start while the
+    previous kernel of the stream still runs, and it would also break the completion chain for the
+    kernel after it."""
+    csrc = os.path.join(ROOT, "paper_2605_05607_b200", "csrc")
+    seen = 0
+    for fn in sorted(os.listdir(csrc)):
+        if not fn.endswith((".cu", ".cuh")):
+            continue
+        text = open(os.path.join(csrc, fn)).read()
+        for m in re.finditer(r"__global__", text):
+            body_start = text.index("{", text.index(")", m.end()))
+            # the body runs to the matching brace
+            depth, i = 0, body_start
+            while True:
+                depth += text[i] == "{"
+                depth -= text[i] == "}"
+                if depth == 0:
+                    break
+                i += 1
+            assert "grid_dependency_sync()" in text[body_start:i], f"{fn}: kernel at offset {m.start()}"
+            seen += 1
+    assert seen >= 15
 
 
 def test_product_package_never_imports_the_oracle():

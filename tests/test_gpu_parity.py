@@ -204,6 +204,14 @@ def test_degenerate_and_error_paths():
     assert st[0] == B.MOE_DEV_INDEX_OUT_OF_RANGE and st[3] == 99
     B.moe_status_reset(run.ws)
     assert run.status()[0] == 0
+    # ... by Combine too: the bad slot (token 3, slot 1) is skipped, the token's other row is still summed
+    assert int(run.lay.pair_row[7]) == -1
+    run.o.copy_(torch.randn(run.o.shape, device="cuda").to(torch.bfloat16))
+    run.combine()
+    st = run.status()
+    assert st[0] == B.MOE_DEV_INDEX_OUT_OF_RANGE and st[1] == B.KERNEL_IDS["combine"] and st[3] == 99, st
+    assert torch.equal(run.y[3], run.o[int(run.lay.pair_row[6])])
+    B.moe_status_reset(run.ws)
 
 
 def test_route_limits_E1024_k32():
@@ -260,13 +268,12 @@ def test_layer_is_capturable_in_a_cuda_graph():
 
 
 @pytest.mark.parametrize("form", ["pair", "single"])
-def test_both_gemm2_forms_on_the_same_layer(form, monkeypatch):
+def test_both_gemm2_forms_on_the_same_layer(form):
     """GEMM-2 has a CTA-pair form (256-row tiles) and a single-CTA form (128-row tiles, taken when experts are
-    small on average); the library picks by shape, TCMOE_GEMM2 forces one.  Both must meet the parity bars on a
-    layer with ragged and empty experts."""
-    monkeypatch.setenv("TCMOE_GEMM2", form)
+    small on average); the library picks by shape, MOE_FLAG_GEMM2_PAIR / MOE_FLAG_GEMM2_SINGLE force one.  Both
+    must meet the parity bars on a layer with ragged and empty experts."""
     cfg = synth.MoEConfig("g2forms", T=1500, d=320, f=448, E=12, k=3, G=4, bias="zipf", zipf_s=1.3, seed=9)
-    staged(cfg)
+    staged(cfg, B.MOE_FLAG_GEMM2_PAIR if form == "pair" else B.MOE_FLAG_GEMM2_SINGLE)
 
 
 def test_bounded_wait_gives_up_and_the_context_stays_usable():

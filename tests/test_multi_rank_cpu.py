@@ -103,3 +103,24 @@ def test_ep_exchange_with_uneven_splits():
     r1 = torch.tensor(res[1][1])
     assert r1.shape == (4, 4) and r1[0, 0] == 12 and r1[1, 0] == 1000 + 16   # rank 0's 4th row, then rank 1's rows 4..
     assert res[0][2] and res[1][2]                                           # the return trip restores the order
+
+
+def test_bench_starts_its_own_ranks_and_reports_the_real_world_size():
+    """`python bench.py --gpus 2` outside a launcher starts two ranks itself; n_gpus in the line is the real
+    world size and the time is the slowest rank's (the stub step of rank r takes (1 + r) ms).  A launcher whose
+    world size disagrees with --gpus is an error, not a silently mislabelled run."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--launcher-selftest", "--gpus", "2",
+                          "--steps", "5"], env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr[-2000:]
+    line = json.loads([ln for ln in out.stdout.splitlines() if ln.startswith("{")][-1])
+    assert line["n_gpus"] == 2 and line["steps"] == 5
+    assert line["ms_per_step"] >= 2.0                                   # rank 1 is the slow one
+    bad = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--launcher-selftest", "--gpus", "2",
+                          "--steps", "1"], env=dict(env, WORLD_SIZE="1", RANK="0"), capture_output=True, text=True,
+                         timeout=300)
+    assert bad.returncode != 0 and "must agree" in bad.stderr
