@@ -325,6 +325,22 @@ int moe_ep_finish(const moe_shape_t* shape, const void* back, const moe_layout_t
  * Reads one int32 from the device and synchronises `stream`.  T = 0 gives zeros. */
 int moe_traffic_stats(const moe_shape_t* shape, const moe_layout_t* layout, double out[8], void* stream);
 
+/* Payload efficiency of one multi-destination transfer under the packet formats of Sec. III-A / III-B
+ * (efficiency = data flits / all transmitted flits, Sec. VI-B).  Host arithmetic only: no device is touched.
+ * What the paper fixes: 16-byte flits; flit0 holds the single multimem address, a stage bit and the target
+ * count; target-extension flits hold eight 16-bit expert ids each; explicit addressing needs one destination
+ * flit per target in the request and as many in the response, which for eight targets lowers an ideal 80 % to
+ * 69 %.  What it leaves open and this library reads as: packets carry at most 256 bytes (16 data flits) and
+ * cost 4 further flits over request and response (the share that makes plain transfers 80 % efficient), and
+ * the destination / target flits are paid once per transfer.  The printed pair 80 % / 69 % is reproduced at
+ * transfer_bytes = 1280, n_targets = 8.
+ *   out[0] data flits = ceil(transfer_bytes / 16)
+ *   out[1] ideal efficiency (headers of plain packets only)
+ *   out[2] explicit addressing: + 2 * n_targets flits
+ *   out[3] dynamic multimem addressing: + ceil(n_targets / 8) flits
+ * transfer_bytes >= 1, 0 <= n_targets < 2^15 (the 15-bit target count), else MOE_ERR_INVALID_ARG. */
+int moe_payload_efficiency(int64_t transfer_bytes, int32_t n_targets, double out[4]);
+
 /* Self-test of the bounded waits every kernel of the library relies on (the paper's runtime polls
  * without a bound, Sec. IV-C; here a wait that outlives its budget ends the kernel with a status
  * instead of hanging the GPU).  Launches one small kernel that waits, with a budget of `limit_ns`

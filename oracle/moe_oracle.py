@@ -308,3 +308,31 @@ def redundancy_figures(D: float, G: int, k: Optional[int] = None) -> Dict[str, f
     return {"allgather_useless": (G - D) / D,
             "redundant_share": (D - 1.0) / (2.0 * D),
             "ideal_speedup": 2.0 * D / (1.0 + D)}
+
+
+# --------------------------------------------------------------------------- packet model
+FLIT_BYTES = 16            # Sec. III-B: the link packet is a sequence of 16-byte flits
+PACKET_DATA_FLITS = 16     # largest payload of one packet: 256 bytes
+PACKET_OVERHEAD_FLITS = 4  # non-data flits per full packet over request + response; the value that makes
+                           # the efficiency of plain (single-destination) transfers the paper's "ideal 80 %"
+IDS_PER_EXTENSION_FLIT = 8 # Sec. III-B: eight 16-bit expert ids per target-extension flit
+
+
+def payload_efficiency(transfer_bytes: int, n_targets: int) -> Dict[str, float]:
+    """Payload efficiency (data flits / all transmitted flits, Sec. VI-B) of one multi-destination
+    transfer of ``transfer_bytes`` under the three addressing schemes of Sec. III-A / III-B:
+
+    * ideal: the transfer cut into packets of at most 256 bytes, each with its fixed header share;
+    * explicit addressing: one destination flit per target in the request and as many again in the
+      response (Sec. III-A: eight GPUs need eight destination flits both ways);
+    * dynamic multimem addressing: the one multimem address stays in flit0 and the target list adds
+      ceil(n_targets / 8) extension flits to the request (Sec. III-B).
+
+    The paper gives the flit counts and the two efficiencies of its example; the fixed header share
+    and the size of that example are not stated (readings, see the constants above)."""
+    data = -(-int(transfer_bytes) // FLIT_BYTES)
+    packets = -(-data // PACKET_DATA_FLITS)
+    base = data + packets * PACKET_OVERHEAD_FLITS
+    explicit = base + 2 * int(n_targets)
+    dynamic = base + -(-int(n_targets) // IDS_PER_EXTENSION_FLIT)
+    return {"data_flits": float(data), "ideal": data / base, "explicit": data / explicit, "dynamic": data / dynamic}

@@ -41,7 +41,8 @@ MOE_FLAG_GEMM2_SINGLE = 64
 EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "moe_status", "moe_strerror",
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",
            "moe_profile_enable", "moe_profile_read", "moe_dispatch_noalloc", "moe_quantize_rows",
-           "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8", "moe_layer_fp8_host", "moe_selftest_wait_timeout", "moe_traffic_stats", "moe_ep_pack", "moe_ep_finish")
+           "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8", "moe_layer_fp8_host", "moe_selftest_wait_timeout", "moe_traffic_stats", "moe_ep_pack", "moe_ep_finish",
+           "moe_payload_efficiency")
 
 
 class MoEShape(ctypes.Structure):
@@ -93,6 +94,7 @@ def lib() -> ctypes.CDLL:
         L.moe_layer_fp8_host.argtypes = [shp, vp, vp, vp, vp, i64, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.moe_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint64, vp]
         L.moe_traffic_stats.argtypes = [shp, lay, ctypes.POINTER(ctypes.c_double), vp]
+        L.moe_payload_efficiency.argtypes = [i64, ctypes.c_int32, ctypes.POINTER(ctypes.c_double)]
         L.moe_ep_pack.argtypes = [shp, vp, vp, lay, vp, vp, vp]
         L.moe_ep_finish.argtypes = [shp, vp, lay, vp, vp]
         L.moe_profile_enable.argtypes = [ctypes.c_int]
@@ -271,6 +273,12 @@ def moe_traffic_stats(shape, layout: Layout, stream=None) -> dict:
     _check("moe_traffic_stats", lib().moe_traffic_stats(ctypes.byref(shape), ctypes.byref(c), out, _stream(stream)))
     names = ("T", "P", "n_disp", "D", "dedup", "allgather_useless", "redundant_share", "ideal_speedup")
     return dict(zip(names, list(out)))
+
+
+def moe_payload_efficiency(transfer_bytes: int, n_targets: int) -> dict:
+    out = (ctypes.c_double * 4)()
+    _check("moe_payload_efficiency", lib().moe_payload_efficiency(transfer_bytes, n_targets, out))
+    return dict(zip(("data_flits", "ideal", "explicit", "dynamic"), list(out)))
 
 
 def moe_selftest_wait_timeout(ws, limit_ns: int, stream=None) -> None:

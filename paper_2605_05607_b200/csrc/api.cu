@@ -262,6 +262,19 @@ int moe_traffic_stats(const moe_shape_t* shape, const moe_layout_t* layout, doub
   return MOE_OK;
 }
 
+int moe_payload_efficiency(int64_t transfer_bytes, int32_t n_targets, double out[4]) {
+  if (out == nullptr || transfer_bytes < 1 || n_targets < 0 || n_targets >= (1 << 15)) return MOE_ERR_INVALID_ARG;
+  constexpr int64_t kFlit = 16, kPacketData = 16, kPacketOverhead = 4, kIdsPerFlit = 8;
+  const int64_t data = (transfer_bytes + kFlit - 1) / kFlit;
+  const int64_t packets = (data + kPacketData - 1) / kPacketData;
+  const int64_t base = data + packets * kPacketOverhead;
+  out[0] = (double)data;
+  out[1] = (double)data / (double)base;
+  out[2] = (double)data / (double)(base + 2 * (int64_t)n_targets);
+  out[3] = (double)data / (double)(base + ((int64_t)n_targets + kIdsPerFlit - 1) / kIdsPerFlit);
+  return MOE_OK;
+}
+
 int moe_selftest_wait_timeout(void* ws, uint64_t limit_ns, void* stream) {
   if (ws == nullptr) return MOE_ERR_INVALID_ARG;
   if (limit_ns < 1000ull || limit_ns > 100000000ull) return MOE_ERR_INVALID_ARG;

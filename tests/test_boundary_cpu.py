@@ -132,6 +132,21 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
         B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"]))
 
 
+def test_payload_efficiency_matches_the_oracle_and_the_printed_pair(lib):
+    """Host-only entry point: the same flit counts as the oracle's packet model on a sweep of sizes and target
+    counts, the paper's printed 80 % -> 69 % (Sec. III-A) at eight targets, bad arguments refused."""
+    from oracle import moe_oracle as O
+    for nbytes in (1, 16, 17, 128, 256, 257, 640, 1280, 4096, 2 * 7168, 2 * 2880):
+        for n in (0, 1, 7, 8, 9, 16, 32):
+            got, ref = B.moe_payload_efficiency(nbytes, n), O.payload_efficiency(nbytes, n)
+            assert got == ref, (nbytes, n, got, ref)
+    r = B.moe_payload_efficiency(1280, 8)
+    assert round(r["ideal"], 2) == 0.80 and round(r["explicit"], 2) == 0.69 and r["explicit"] < r["dynamic"] < r["ideal"]
+    for bad in ((0, 8), (-5, 1), (256, -1), (256, 1 << 15)):
+        with pytest.raises(B.MoEError):
+            B.moe_payload_efficiency(*bad)
+
+
 def test_every_kernel_waits_for_its_stream_predecessor():
     """All kernels are launched with programmatic stream serialisation, so each must call
     grid_dependency_sync() before it touches global memory: a kernel without it could start while the

@@ -466,3 +466,26 @@ def test_config_dedup_statistics_match_closed_form():
         idx, _ = O.route(logits, None, cfg.k, cfg.score_fn)
         D = O.distinct_groups_per_token(idx, cfg.E, cfg.G)
         assert D == pytest.approx(closed_form_D(cfg.E, cfg.G, cfg.k), rel=0.03)
+
+
+def test_payload_efficiency_reproduces_the_papers_printed_pair(golden_dir):
+    """Sec. III-A prints one worked example of the packet model: eight targets, explicit addressing, ideal 80 % ->
+    69 %.  The oracle must print the same two figures, keep the multimem-style format near the ideal, and obey the
+    closed forms of the flit count (hand-computed below, not re-typed from the function)."""
+    gold = json.load(open(os.path.join(golden_dir, "paper_payload_efficiency.json")))
+    r = O.payload_efficiency(gold["transfer_bytes_of_the_printed_pair"], gold["n_targets"])
+    assert round(r["ideal"], gold["printed_digits"]) == gold["ideal"]
+    assert round(r["explicit"], gold["printed_digits"]) == gold["explicit"]
+    assert r["explicit"] < r["dynamic"] < r["ideal"] and r["ideal"] - r["dynamic"] < 0.01      # "near-ideal"
+    # hand count: 1280 B = 80 data flits in 5 packets -> 20 header flits; explicit +16; multimem-style +1
+    assert r["data_flits"] == 80 and abs(r["explicit"] - 80 / 116) < 1e-15 and abs(r["dynamic"] - 80 / 101) < 1e-15
+    # one target costs one extension flit, nine targets two; a single 16-byte flit still pays a whole header
+    assert O.payload_efficiency(256, 1)["dynamic"] == 16 / 21 and O.payload_efficiency(256, 9)["dynamic"] == 16 / 22
+    assert O.payload_efficiency(16, 0)["ideal"] == 1 / 5 and O.payload_efficiency(17, 0)["data_flits"] == 2
+    # a token vector of the DeepSeek-V3-shaped layer (7168 bf16): the header share vanishes, all three converge
+    big = O.payload_efficiency(7168 * 2, 8)
+    assert big["ideal"] == 0.8 and abs(big["explicit"] - 896 / 1136) < 1e-15 and big["explicit"] < big["dynamic"] < 0.8
+    # efficiency never decreases when targets are removed
+    for n in range(1, 33):
+        a, b = O.payload_efficiency(640, n), O.payload_efficiency(640, n - 1)
+        assert a["explicit"] < b["explicit"] and a["dynamic"] <= b["dynamic"]
