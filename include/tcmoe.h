@@ -80,23 +80,37 @@ enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1,   /* default (0): gate weight applied in 
                                             number of slots in use (<= T*k), pair_row is -1 for
                                             unused slots, and the per-pair arrays are filled only
                                             up to expert_offsets[E].                          */
-       MOE_FLAG_SM_PARTITION = 16,       /* with MOE_FLAG_FUSED_FFN: the thread blocks are divided
-                                            between the stages as in Sec. IV - two thirds of the
-                                            SMs take only GEMM-1 tiles, one third only GEMM-2
-                                            tiles, the second group paced by the tracker alone.
-                                            Same results.                                      */
+       MOE_FLAG_SM_PARTITION = 16,       /* with MOE_FLAG_FUSED_FFN: the thread blocks are divided between the
+                                            stages as in Sec. IV-C - two thirds of the SMs take only GEMM-1 tiles
+                                            (their worker warps the Dispatch tasks), one third only GEMM-2 tiles
+                                            (their worker warps the Combine tasks), each group paced by the tracker
+                                            alone.  Same results.                                                 */
+       MOE_FLAG_GEMM1_PAIR = 128,        /* moe_expert_ffn / moe_layer (bf16 experts): Dispatch writes the per-expert
+                                            layout tensors of Sec. III-D (one dense row per (token, expert), expert-
+                                            sorted, in the workspace) and GEMM-1 reads them as TMA tiles on CTA pairs
+                                            (cta_group::2, 256-row tiles) instead of gathering token rows inside
+                                            the GEMM.  Same h as the gathering form.  Excludes MOE_FLAG_FUSED_FFN.     */
+       MOE_FLAG_TRACK_DISPATCH = 256,    /* with MOE_FLAG_FUSED_FFN: Dispatch runs as tasks of the same kernel.  Worker
+                                            warps write the per-expert layout tensors (Sec. III-D) 16 rows at a time and
+                                            count them in the Tile Status table (DAcc, Sec. IV-B); a GEMM-1 tile starts
+                                            when all rows of its 128-row tile have landed and reads them in place.
+                                            Without the flag GEMM-1 gathers token rows itself and no copy is written.
+                                            Same results.                                                          */
        MOE_FLAG_GEMM2_PAIR = 32,         /* GEMM-2 runs on 256-row CTA-pair tiles (cta_group::2) whatever the shape */
        MOE_FLAG_GEMM2_SINGLE = 64,       /* GEMM-2 runs on 128-row single-CTA tiles whatever the shape.  Without either
                                             flag the library picks from the shape: pair tiles unless experts hold
                                             fewer than 512 rows on average.  The two flags exclude each other; the
                                             results of both forms meet the same tolerances.               */
-       MOE_FLAG_FUSED_FFN = 8 };         /* moe_expert_ffn / moe_layer (bf16 experts): GEMM-1 and
-                                            GEMM-2 run as ONE persistent kernel paced by a tile
-                                            tracker (Sec. IV token-centric kernel fusion, tiles of
-                                            128 tokens): a GEMM-2 tile starts as soon as the
-                                            128 rows of h it reads are complete.  Same results as
-                                            the two-kernel form (bit for bit); excludes
-                                            MOE_FLAG_COMBINE_IN_EPILOGUE.                      */
+       MOE_FLAG_FUSED_FFN = 8 };         /* moe_expert_ffn / moe_layer (bf16 experts): the stages after the layout run
+                                            as ONE persistent kernel paced by the token tracker of Sec. IV-B (tiles of
+                                            128 tokens): a GEMM-2 tile starts as soon as the 128 rows of h it reads are
+                                            complete (TBCnt1); in moe_layer the kernel also runs the Combine tasks - a
+                                            token is combined when all of its topk rows of o are complete (TBCnt2 and
+                                            the Output Readiness counter nReady), so y is produced by the same launch.
+                                            Same results as the separate kernels, bit for bit.  Excludes
+                                            MOE_FLAG_COMBINE_IN_EPILOGUE.  The kernel needs every thread block of its
+                                            grid resident at once (one per SM): a device shared with other work may
+                                            make its bounded waits expire (MOE_DEV_TIMEOUT after 2 s), never hang.   */
 
 /* Shape of one layer.  Limits: 1 <= k <= min(E, 32); E <= 1024; E % G == 0;
  * d % 8 == 0; f % 8 == 0; T >= 0; T * max(k, G) < 2^31. */

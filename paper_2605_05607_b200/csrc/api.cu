@@ -18,7 +18,7 @@ inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 // Regions of the workspace, in order.  Every region starts on a 1 KiB boundary.
 struct WsPlan {
-  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, blk_start, blk_info, n_blocks, done, wsplit, h, hq, sh, xq, sx, o, logits, topk_idx, topk_w;
+  size_t status, emask, gmask, eprefix, gprefix, mt_prefix, mp_prefix, blk_start, blk_info, n_blocks, tracker, wsplit, xs, h, hq, sh, xq, sx, o, logits, topk_idx, topk_w;
   size_t expert_counts, expert_offsets, group_counts, group_offsets, pair_row, row_pair, al, disp_token, row_src;
   size_t total;
   int W;
@@ -51,9 +51,11 @@ WsPlan plan(const moe_shape_t& s) {
     p.blk_start = take(3 * (nbmax + 1) * 4);   // interleaved | GEMM-1 only | GEMM-2 only
     p.blk_info = take(3 * (nbmax + 1) * 16);
     p.n_blocks = take(3 * 4);
-    p.done = take((P / 128 + E + 1) * 4);
+    p.tracker = take(fused_tracker_bytes(Shape{s.T, s.d, s.f, s.E, s.k, s.G, s.score_fn, s.flags}));
   }
   p.wsplit = take(gate_split_bytes(s.d, s.E));
+  // expert-sorted activation rows of the CTA-pair GEMM-1 (only reserved when that form is asked for)
+  p.xs = take((s.flags & (MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH)) ? P * (size_t)s.d * 2 : 0);
   p.h = take(P * (size_t)s.f * 2);
   p.hq = take(P * (size_t)s.f);   // FP8 form: E4M3 copy of h and its row scales
   p.sh = take(P * 4);
@@ -82,10 +84,12 @@ int check_shape(const moe_shape_t* s) {
   if (s->T < 0 || s->d <= 0 || s->f <= 0 || s->E <= 0 || s->k <= 0 || s->G <= 0) return MOE_ERR_INVALID_ARG;
   if (s->score_fn != MOE_SCORE_SOFTMAX && s->score_fn != MOE_SCORE_SIGMOID) return MOE_ERR_INVALID_ARG;
   if (s->flags & ~(MOE_FLAG_WEIGHT_IN_COMBINE | MOE_FLAG_COMBINE_IN_EPILOGUE | MOE_FLAG_SPARSE_TOPK | MOE_FLAG_FUSED_FFN |
-                   MOE_FLAG_SM_PARTITION | MOE_FLAG_GEMM2_PAIR | MOE_FLAG_GEMM2_SINGLE))
+                   MOE_FLAG_SM_PARTITION | MOE_FLAG_GEMM2_PAIR | MOE_FLAG_GEMM2_SINGLE | MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH))
     return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_GEMM2_PAIR) && (s->flags & MOE_FLAG_GEMM2_SINGLE)) return MOE_ERR_INVALID_ARG;
+  if ((s->flags & MOE_FLAG_GEMM1_PAIR) && (s->flags & MOE_FLAG_FUSED_FFN)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_SM_PARTITION) && !(s->flags & MOE_FLAG_FUSED_FFN)) return MOE_ERR_INVALID_ARG;
+  if ((s->flags & MOE_FLAG_TRACK_DISPATCH) && !(s->flags & MOE_FLAG_FUSED_FFN)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_FUSED_FFN) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_WEIGHT_IN_COMBINE) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
   if (s->k > s->E || s->G > s->E || s->E % s->G != 0) return MOE_ERR_INVALID_ARG;
@@ -425,6 +429,8 @@ int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t*
   a.w1 = w1;
   a.w3 = w3;
   a.w2 = w2;
+  a.xs = (shape->flags & (MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH)) ? at<void>(ws, p.xs) : nullptr;
+  a.track_dispatch = (shape->flags & MOE_FLAG_TRACK_DISPATCH) != 0;
   a.h = at<void>(ws, p.h);
   a.o = o;
   a.topk_w = in_combine ? nullptr : topk_w;
@@ -436,7 +442,7 @@ int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t*
   a.blk_start = at<int32_t>(ws, p.blk_start);
   a.blk_info = at<void>(ws, p.blk_info);
   a.n_blocks = at<int32_t>(ws, p.n_blocks);
-  a.done = at<int32_t>(ws, p.done);
+  a.tracker = at<int32_t>(ws, p.tracker);
   a.status = at<int32_t>(ws, p.status);
   // rebuilt from the counts so that this call does not depend on what moe_dispatch left in ws
   TCMOE_CUDA(launch_tile_prefix(to_shape(*shape), layout->expert_counts, at<int32_t>(ws, p.mt_prefix),
@@ -492,6 +498,8 @@ int moe_expert_ffn_fp8(const moe_shape_t* shape, const void* xq, const float* sx
   a.w1 = w1q;
   a.w3 = w3q;
   a.w2 = w2q;
+  a.xs = (shape->flags & (MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH)) ? at<void>(ws, p.xs) : nullptr;
+  a.track_dispatch = (shape->flags & MOE_FLAG_TRACK_DISPATCH) != 0;
   a.h = at<void>(ws, p.h);
   a.o = o;
   a.topk_w = in_combine ? nullptr : topk_w;
@@ -503,7 +511,7 @@ int moe_expert_ffn_fp8(const moe_shape_t* shape, const void* xq, const float* sx
   a.blk_start = at<int32_t>(ws, p.blk_start);
   a.blk_info = at<void>(ws, p.blk_info);
   a.n_blocks = at<int32_t>(ws, p.n_blocks);
-  a.done = at<int32_t>(ws, p.done);
+  a.tracker = at<int32_t>(ws, p.tracker);
   a.status = at<int32_t>(ws, p.status);
   Fp8Args q{sx, s1, s3, s2, at<void>(ws, p.hq), at<float>(ws, p.sh)};
   cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -597,6 +605,8 @@ static int layer_impl(const moe_shape_t* shape, const void* x, const float* w_ga
   a.w1 = w1;
   a.w3 = w3;
   a.w2 = w2;
+  a.xs = (shape->flags & (MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH)) ? at<void>(ws, p.xs) : nullptr;
+  a.track_dispatch = (shape->flags & MOE_FLAG_TRACK_DISPATCH) != 0;
   a.h = at<void>(ws, p.h);
   a.o = at<void>(ws, p.o);
   a.topk_w = (s.flags & MOE_FLAG_WEIGHT_IN_COMBINE) ? nullptr : tw;
@@ -608,7 +618,7 @@ static int layer_impl(const moe_shape_t* shape, const void* x, const float* w_ga
   a.blk_start = at<int32_t>(ws, p.blk_start);
   a.blk_info = at<void>(ws, p.blk_info);
   a.n_blocks = at<int32_t>(ws, p.n_blocks);
-  a.done = at<int32_t>(ws, p.done);
+  a.tracker = at<int32_t>(ws, p.tracker);
   a.status = status;
   if (s.flags & MOE_FLAG_COMBINE_IN_EPILOGUE) {
     // o never materialises: GEMM-2 adds each weighted row into its token's fp32 accumulator
@@ -616,6 +626,15 @@ static int layer_impl(const moe_shape_t* shape, const void* x, const float* w_ga
     if (s.T > 0) TCMOE_CUDA(cudaMemsetAsync(a.y_acc, 0, (size_t)s.T * s.d * 4, st));
     TCMOE_CUDA(fp8 != nullptr ? launch_expert_ffn_fp8(s, a, q, st) : launch_expert_ffn(s, a, st));
     TCMOE_CUDA(launch_round_rows(s, a.y_acc, y, st));
+    return MOE_OK;
+  }
+  if (s.flags & MOE_FLAG_FUSED_FFN) {
+    // one kernel after the layout: GEMM-1, GEMM-2 and Combine tasks (and Dispatch tasks when asked for) paced by
+    // the token tracker; the Combine tasks produce y
+    a.comb = CombineArgs{static_cast<const uint4*>(a.o), static_cast<uint4*>(y), nullptr, idx, tw, L.pair_row, L.al,
+                         L.group_offsets, s.T, s.E, s.k, s.E / s.G, s.d / 8,
+                         (s.flags & MOE_FLAG_WEIGHT_IN_COMBINE) ? 1 : 0, s.T * s.k, status};
+    TCMOE_CUDA(launch_expert_ffn(s, a, st));
     return MOE_OK;
   }
   TCMOE_CUDA(fp8 != nullptr ? launch_expert_ffn_fp8(s, a, q, st) : launch_expert_ffn(s, a, st));

@@ -59,6 +59,20 @@ struct Layout {
       *disp_token, *row_src;
 };
 
+// Arguments of the Combine stage (the combine kernel and the Combine tasks of the tracker-paced kernel).
+struct CombineArgs {
+  const uint4* o;                 // [P, d] bf16 expert-sorted rows
+  uint4* y;                       // [T, d] bf16 out
+  uint4* pg;                      // NULL or [N_disp, d] bf16 out (group partial sums)
+  const int32_t* topk_idx;        // [T, k]
+  const float* topk_w;            // [T, k] (read only when weighted)
+  const int32_t* pair_row;        // [T, k]
+  const int32_t* al;              // [G, T]
+  const int32_t* group_offsets;   // [G + 1]
+  int T, E, k, m, vec_per_row, weighted, n_rows;
+  int32_t* status;
+};
+
 // Scratch tables of the layout builder (inside the workspace).
 struct LayoutScratch {
   uint32_t* emask;    // [E, W] bit t%32 of word t/32: token t selected expert e
@@ -84,6 +98,9 @@ cudaError_t launch_layout(const Shape& s, const int32_t* topk_idx, const Layout&
 cudaError_t launch_tile_prefix(const Shape& s, const int32_t* expert_counts, int32_t* mt_prefix, int32_t* mp_prefix,
                                cudaStream_t st);
 cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void* xg, cudaStream_t st);
+cudaError_t launch_permute_rows(const Shape& s, const void* src, int src_rows, const int32_t* gather_idx,
+                                int gather_div, const int32_t* expert_offsets, void* xs, int32_t* status,
+                                cudaStream_t st);
 cudaError_t launch_round_rows(const Shape& s, const float* acc, void* y, cudaStream_t st);
 cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
                            const float* topk_w, void* pg, void* y, int32_t* status, cudaStream_t st);
@@ -94,6 +111,7 @@ struct FfnArgs {
   const int32_t* gather_idx;  // row_src, or row_pair (token = row_pair / k)
   int gather_div;
   const void *w1, *w3, *w2;
+  void* xs;                   // [P, d] bf16 scratch: expert-sorted activation rows (CTA-pair GEMM-1), or NULL
   void* h;                    // [P, f] bf16 scratch
   void* o;                    // [P, d] bf16 out (unused when y_acc is set)
   float* y_acc;               // Combine in GEMM-2's epilogue: zeroed fp32 [T, d] accumulator, else NULL
@@ -107,10 +125,13 @@ struct FfnArgs {
   int32_t* blk_start;
   void* blk_info;
   int32_t* n_blocks;
-  int32_t* done;
+  int32_t* tracker;           // fused_tracker_words() int32 words
+  CombineArgs comb;           // comb.y != NULL: the kernel also runs the Combine tasks (moe_layer)
+  bool track_dispatch;        // Dispatch tasks write xs inside the kernel, GEMM-1 waits for them (needs xs)
   int32_t* status;
 };
 size_t fused_table_blocks(const Shape& s);   // task-block capacity for a shape (ffn_fused.cu)
+size_t fused_tracker_bytes(const Shape& s);  // bytes of the tracker tables for a shape
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st);
 // FP8 form of the expert FFN: a.a_src / a.w1 / a.w3 / a.w2 hold E4M3 codes (weights [E, N, K]).
 struct Fp8Args {

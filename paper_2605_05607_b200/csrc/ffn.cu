@@ -111,6 +111,7 @@ static bool small_experts(const Shape& s) {
 }
 
 size_t fused_table_blocks(const Shape& s) { return ffn::fused_max_blocks(s.T, s.k, s.E); }
+size_t fused_tracker_bytes(const Shape& s) { return ffn::fused_tracker_words(s.T, s.k, s.E) * sizeof(int32_t); }
 
 // flag bit 8 (MOE_FLAG_FUSED_FFN): both GEMMs in one persistent kernel paced by the tile tracker
 static cudaError_t launch_expert_ffn_fused(const Shape& s, const FfnArgs& a, cudaStream_t st) {
@@ -136,16 +137,18 @@ static cudaError_t launch_expert_ffn_fused(const Shape& s, const FfnArgs& a, cud
   p.tbl_stride = (int)fused_table_blocks(s) + 1;
   // flag bit 16 (MOE_FLAG_SM_PARTITION): two thirds of the SMs for GEMM-1 (it has two thirds of the flops)
   p.part_g1 = (s.flags & 16) ? (2 * sm_count() + 1) / 3 : 0;
-  p.done = a.done;
   p.E = s.E;
   p.d = s.d;
   p.f = s.f;
+  p.T = s.T;
+  p.k = s.k;
   p.n1 = (s.f + 127) / 128;
   p.n2 = (s.d + 255) / 256;
   p.status = a.status;
-  const size_t done_entries = (size_t)s.T * s.k / ffn::BM + s.E + 1;
-  return ffn::launch_ffn_fused(p, a.expert_counts, a.blk_start, static_cast<int4*>(a.blk_info), a.n_blocks,
-                               done_entries, m_w1, m_w3, m_w2, st);
+  p.comb = a.comb;                                        // comb.y == NULL: no Combine tasks
+  p.xs = a.track_dispatch ? static_cast<__nv_bfloat16*>(a.xs) : nullptr;   // NULL: no Dispatch tasks
+  return ffn::launch_ffn_fused(p, a.expert_counts, a.blk_start, static_cast<int4*>(a.blk_info), a.n_blocks, a.tracker,
+                               m_w1, m_w3, m_w2, st);
 }
 
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st) {
@@ -172,7 +175,19 @@ cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st)
   g1.N = s.f;
   g1.n_tiles = (s.f + 127) / 128;
   g1.status = a.status;
-  cudaError_t err = ffn::launch_gemm1(g1, m_w1, m_w3, false, st);
+  cudaError_t err;
+  if ((s.flags & 128) && a.xs != nullptr) {
+    // flag bit 128 (MOE_FLAG_GEMM1_PAIR): Dispatch writes the per-expert layout tensors, GEMM-1 runs on CTA pairs
+    CUtensorMap m_xs;
+    if (!make_act_map(&m_xs, a.xs, P, s.d)) return cudaErrorInvalidValue;
+    if ((err = launch_permute_rows(s, a.a_src, a.a_rows, a.gather_idx, a.gather_div, a.expert_offsets, a.xs, a.status,
+                                   st)) != cudaSuccess)
+      return err;
+    g1.tile_prefix = a.mp_prefix;
+    err = ffn::launch_gemm1_pair(g1, m_w1, m_w3, m_xs, st);
+  } else {
+    err = ffn::launch_gemm1(g1, m_w1, m_w3, false, st);
+  }
   if (err != cudaSuccess) return err;
 
   ffn::GemmParams g2{};

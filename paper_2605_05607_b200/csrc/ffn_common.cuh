@@ -1,6 +1,7 @@
 // Pieces shared by the two expert-FFN GEMM kernels (paper Sec. II-A GEMM-1 / GEMM-2): tile
 // geometry, the device-side task decode, UMMA descriptors and small epilogue helpers.
 #pragma once
+#include "combine.cuh"
 #include "common.cuh"
 #include "ptx.cuh"
 
@@ -104,7 +105,7 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// Parameters of the single-kernel FFN (ffn_fused.cu)
+// Parameters of the tracker-paced kernel (ffn_fused.cu)
 struct FusedParams {
   const void* x;                // GEMM-1 gather source (xg or x), bf16
   int x_ld;
@@ -123,7 +124,16 @@ struct FusedParams {
   const int32_t* n_blocks;      // [3] device scalars
   int tbl_stride;
   int part_g1;                  // SM partition: CTAs [0, part_g1) take GEMM-1 tiles, the rest GEMM-2 tiles; 0: none
-  int32_t* done;                // tracker: parts stored per 128-row tile of h (zeroed before the launch)
+  // Tracker (Sec. IV-B), all zeroed before the launch.  Tile Status table, one entry per 128-row tile:
+  int32_t* dacc;                //   DAcc   rows of the tile that Dispatch has written (NULL: no Dispatch tasks)
+  int32_t* done;                //   TBCnt1 parts of the h tile stored by GEMM-1 (4 warps x n1 column tiles)
+  int32_t* tbcnt2;              //   TBCnt2 parts of the o tile stored by GEMM-2 (4 warps x n2 column tiles)
+  int32_t* nready;              // Output Readiness table: complete rows of o per token (NULL: no Combine tasks)
+  int32_t* queue;               // [2] next Dispatch unit, next Combine chunk (work handed out in order)
+  __nv_bfloat16* xs;            // per-expert layout tensors [P, d] written by the Dispatch tasks (with dacc)
+  CombineArgs comb;             // Combine tasks (with nready)
+  int T, k;
+  int chunk_tokens;             // tokens per Combine chunk (1..32)
   int E, d, f, n1, n2;          // n1 = ceil(f / 128) GEMM-1 column tiles, n2 = ceil(d / 256) GEMM-2 column tiles
   int32_t* status;
 };
@@ -138,9 +148,12 @@ cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUt
                          cudaStream_t st);
 cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, bool fp8,
                          cudaStream_t st);
+cudaError_t launch_gemm1_pair(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3,
+                              const CUtensorMap& m_xs, cudaStream_t st);
 size_t fused_max_blocks(int T, int k, int E);   // capacity of blk_start (+1) / blk_info for a shape
-cudaError_t launch_ffn_fused(const FusedParams& p, const int32_t* expert_counts, int32_t* blk_start, int4* blk_info,
-                             int32_t* n_blocks, size_t done_entries, const CUtensorMap& m_w1, const CUtensorMap& m_w3,
+size_t fused_tracker_words(int T, int k, int E);   // int32 words of the tracker region (dacc | done | tbcnt2 | nready | queue)
+cudaError_t launch_ffn_fused(FusedParams p, const int32_t* expert_counts, int32_t* blk_start, int4* blk_info,
+                             int32_t* n_blocks, int32_t* tracker, const CUtensorMap& m_w1, const CUtensorMap& m_w3,
                              const CUtensorMap& m_w2, cudaStream_t st);
 // GEMM-2 on 128-row single-CTA tiles (small experts): p.a_src / p.a_ld = h rows, no Combine-in-epilogue form
 cudaError_t launch_gemm2_single(const GemmParams& p, const CUtensorMap& m_w2, bool fp8, cudaStream_t st);

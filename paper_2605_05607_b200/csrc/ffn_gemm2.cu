@@ -3,6 +3,12 @@
 // un-weighted reduction):
 //     o[r, n] = w_r * (h_r . W2[e][:, n])
 //
+// The same kernel, with GLU = true, is the CTA-pair form of GEMM-1 (Sec. II-A "GEMM-1") on rows that Dispatch
+// has already placed in expert-sorted order (the per-expert layout tensors of Sec. III-D):
+//     h[r, n] = silu(a_r . W1[e][:, n]) * (a_r . W3[e][:, n])
+// CTA 0 of the pair then holds the 128-column tile of W1 and CTA 1 the same tile of W3, so the pair's 256
+// accumulator columns are [a.W1 | a.W3] for every row and the epilogue applies SwiGLU to column c and c + 128.
+//
 // Both operands come by TMA (h rows are contiguous in expert-sorted order).  CTAs work in pairs
 // (cluster of 2, tcgen05 cta_group::2): each CTA holds 128 rows of h and one half of the
 // 256-column W2 tile; one UMMA of M = 256 spans the pair, so every weight byte is fetched and read
@@ -37,7 +43,6 @@ constexpr int COLSCALE_WARP = UMMA_N * 4;          // FP8: one warp's copy of th
 constexpr int SMEM_BYTES =
     1024 + NSTAGE * STAGE_BYTES + NUM_BARS * 8 + 64 + TABLE_BYTES + 4 * STAGE_OUT_WARP + 4 * COLSCALE_WARP;
 constexpr int THREADS = 192;
-constexpr int BN_OUT = 256;
 constexpr uint32_t IDESC = idesc_bf16(2 * BM);
 constexpr uint32_t IDESC_F8 = idesc_e4m3(2 * BM);
 constexpr uint32_t HINT = 4000;   // try_wait suspend-time hint (ns), see ptx::mbar_try_wait
@@ -48,10 +53,14 @@ constexpr uint32_t HINT = 4000;   // try_wait suspend-time hint (ns), see ptx::m
 // FP8 = true: h rows and weights are E4M3 codes, a stage holds 128 elements of K (the same 128 bytes
 // per row), W2 comes K-major from [E, N, K] as one 128-row box per CTA, and the epilogue applies
 // a_scale[row] * b_scale[e, n] together with the gate weight.
-template <bool RED, bool FP8>
+// GLU = true: GEMM-1 with the SwiGLU epilogue (see the head of this file): map_b0 = W1, map_b1 = W3, 128 output
+// columns per tile; otherwise map_b0 = map_b1 = W2 and CTA `rank` takes columns n0 + 128 * rank.
+template <bool RED, bool FP8, bool GLU>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
-ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_constant__ CUtensorMap map_h,
-                 const GemmParams p) {
+ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
+                 const __grid_constant__ CUtensorMap map_h, const GemmParams p) {
+  static_assert(!(GLU && (RED || FP8)), "the SwiGLU form exists for bf16 operands and row output only");
+  constexpr int BN_OUT = GLU ? 128 : 256;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + NSTAGE * STAGE_BYTES);
@@ -85,7 +94,8 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
     ptx::fence_mbar_init();
   }
   if (warp == 4 && lane == 0) {
-    ptx::prefetch_tensormap(&map_w2);
+    ptx::prefetch_tensormap(&map_b0);
+    ptx::prefetch_tensormap(&map_b1);
     ptx::prefetch_tensormap(&map_h);
   }
   if (warp == 5) {
@@ -110,7 +120,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
   const volatile int* global_abort = p.status + ST_ABORT;
 
   auto timeout = [&](int detail) {
-    report_error(p.status, DEV_TIMEOUT, KID_GEMM2, detail, blockIdx.x);
+    report_error(p.status, DEV_TIMEOUT, GLU ? KID_GEMM1 : KID_GEMM2, detail, blockIdx.x);
     p.status[ST_ABORT] = 1;
     *abort_flag = 1;
   };
@@ -130,7 +140,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UMMA_N);
       float* yrow = nullptr;
       float wr = 1.f;
-      if (valid) {
+      if (valid && !GLU) {
         const int pair = __ldg(p.row_pair + grow);
         if (p.topk_w != nullptr) wr = __ldg(p.topk_w + pair);
         if (FP8) wr *= __ldg(p.a_scale + grow);   // row scale of h joins the gate weight
@@ -148,7 +158,45 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
         }
         __syncwarp();
       }
-      if (RED) {
+      if (GLU) {
+        // SwiGLU of the W1 half (columns 0..127) and the W3 half (128..255): 128 columns of h, transposed
+        // through shared memory 64 columns at a time and stored as whole 128-byte row segments
+        const uint32_t stage = stage_base + (uint32_t)(warp * STAGE_OUT_WARP);
+        const int srow = lane >> 3, piece = lane & 7;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t a1[32], a3[32];
+          ptx::tmem_ld32(taddr + c * 32, a1);
+          ptx::tmem_ld32(taddr + 128 + c * 32, a3);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int v = 0; v < 4; ++v) {
+            uint32_t q[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const int j = v * 8 + 2 * i;
+              q[i] = pack2(silu_mul(__uint_as_float(a1[j]), __uint_as_float(a3[j])),
+                           silu_mul(__uint_as_float(a1[j + 1]), __uint_as_float(a3[j + 1])));
+            }
+            ptx::st_shared_v4(stage + lane * 144 + (c & 1) * 64 + v * 16, q[0], q[1], q[2], q[3]);
+          }
+          if (c & 1) {
+            __syncwarp();
+            const int col = t.n0 + (c - 1) * 32 + piece * 8;
+            if (col < p.N) {
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const int r = i * 4 + srow;
+                if (warp * 32 + r < t.rows) {
+                  const uint4 q = ptx::ld_shared_v4(stage + r * 144 + piece * 16);
+                  *reinterpret_cast<uint4*>(p.out + (size_t)(t.row0 + warp * 32 + r) * (size_t)p.out_ld + col) = q;
+                }
+              }
+            }
+            __syncwarp();
+          }
+        }
+      } else if (RED) {
 #pragma unroll 1
         for (int c = 0; c < 8; ++c) {
           uint32_t acc[32];
@@ -250,11 +298,13 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_w2, const __grid_consta
           if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
           const int k0 = kb * BK_ELEMS;
           ptx::tma_load_2d_pair(sa, &map_h, lead_full, k0, t.row0);
+          const CUtensorMap* map_b = rank == 0 ? &map_b0 : &map_b1;
+          const int nb = GLU ? t.n0 : t.n0 + rank * 128;   // this CTA's 128 columns of the B tile
           if (FP8) {   // one K-major box: this CTA's 128 output columns x 128 bytes of K
-            ptx::tma_load_3d_pair(sb, &map_w2, lead_full, k0, t.n0 + rank * 128, t.e);
+            ptx::tma_load_3d_pair(sb, map_b, lead_full, k0, nb, t.e);
           } else {     // two MN-major slabs of 64 output columns x 64 rows of K
-            ptx::tma_load_3d_pair(sb, &map_w2, lead_full, t.n0 + rank * 128, k0, t.e);
-            ptx::tma_load_3d_pair(sb + 8192, &map_w2, lead_full, t.n0 + rank * 128 + 64, k0, t.e);
+            ptx::tma_load_3d_pair(sb, map_b, lead_full, nb, k0, t.e);
+            ptx::tma_load_3d_pair(sb + 8192, map_b, lead_full, nb + 64, k0, t.e);
           }
         }
         if (!ok) break;
@@ -330,7 +380,7 @@ int pair_grid() {
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    if (cudaOccupancyMaxActiveClusters(&clusters, ffn_gemm2_kernel<false, false>, &cfg) != cudaSuccess || clusters <= 0) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, ffn_gemm2_kernel<false, false, false>, &cfg) != cudaSuccess || clusters <= 0) {
       (void)cudaGetLastError();
       clusters = sm_count() / 2;
     }
@@ -342,28 +392,47 @@ int pair_grid() {
 
 }  // namespace
 
-cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, bool fp8,
-                         cudaStream_t st) {
+namespace {
+cudaError_t set_pair_attributes() {
   // per device; several host threads may get here at once: setting the attribute twice is harmless
   static std::atomic<bool> attr_set[MAX_DEVICES];
   const int dev = current_device();
   if (!attr_set[dev].load(std::memory_order_acquire)) {
     const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false>, attr, SMEM_BYTES);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, false>, attr, SMEM_BYTES);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, true>, attr, SMEM_BYTES);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, true>, attr, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, false, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, true, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, true, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, true>, attr, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set[dev].store(true, std::memory_order_release);
   }
+  return cudaSuccess;
+}
+}  // namespace
+
+cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUtensorMap& m_h, bool fp8,
+                         cudaStream_t st) {
+  cudaError_t e = set_pair_attributes();
+  if (e != cudaSuccess) return e;
   ProfileScope prof(KID_GEMM2, st);
   const bool red = p.y_acc != nullptr;
   if (fp8) {
-    if (red) return launch_pdl(ffn_gemm2_kernel<true, true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
-    return launch_pdl(ffn_gemm2_kernel<false, true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
+    if (red) return launch_pdl(ffn_gemm2_kernel<true, true, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, p);
+    return launch_pdl(ffn_gemm2_kernel<false, true, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, p);
   }
-  if (red) return launch_pdl(ffn_gemm2_kernel<true, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
-  return launch_pdl(ffn_gemm2_kernel<false, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_h, p);
+  if (red) return launch_pdl(ffn_gemm2_kernel<true, false, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, p);
+  return launch_pdl(ffn_gemm2_kernel<false, false, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, p);
+}
+
+// GEMM-1 on CTA pairs: m_xs maps the expert-sorted activation rows [P, K]; p.tile_prefix = the 256-row pair-tile
+// prefix, p.n_tiles = ceil(N / 128), p.out = h.
+cudaError_t launch_gemm1_pair(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3,
+                              const CUtensorMap& m_xs, cudaStream_t st) {
+  cudaError_t e = set_pair_attributes();
+  if (e != cudaSuccess) return e;
+  ProfileScope prof(KID_GEMM1, st);
+  return launch_pdl(ffn_gemm2_kernel<false, false, true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w1, m_w3, m_xs, p);
 }
 
 }  // namespace ffn

@@ -7,9 +7,7 @@
 // (one bit per (expert, token) and per (group, token)) are built with order-independent atomicOr,
 // an exclusive popcount scan along each mask row gives every token its rank, and a fill pass
 // turns ranks into the row tables.  No atomics touch the result arrays.
-#include "common.cuh"
-
-#include <cuda_bf16.h>
+#include "combine.cuh"
 
 namespace tcmoe {
 
@@ -226,6 +224,57 @@ __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__
   }
 }
 
+// ---- K3b: dispatch into the per-expert layout tensors ----------------------------------------------
+// xs[r, :] = src[gather_idx[r] / gather_div, :] for every expert-sorted row r: the dense per-expert buffers that
+// the destination's memory manager fills in the paper (Sec. III-D: one AL sub-table per local expert), which is
+// what lets GEMM-1 read its rows as plain TMA tiles.  One warp per row, 16-byte vectors; the number of rows in
+// use is read from the device (expert_offsets[E]).
+__global__ void __launch_bounds__(256) permute_rows_kernel(const uint4* __restrict__ src, uint4* __restrict__ xs,
+                                                           const int32_t* __restrict__ gather_idx, int gather_div,
+                                                           const int32_t* __restrict__ expert_offsets, int E,
+                                                           int src_rows, int vec_per_row, int32_t* status) {
+  grid_dependency_sync();
+  const int lane = threadIdx.x & 31;
+  const int wpb = blockDim.x >> 5;
+  const int rows = __ldg(expert_offsets + E);
+  for (int r = blockIdx.x * wpb + (threadIdx.x >> 5); r < rows; r += gridDim.x * wpb) {
+    int idx = __ldg(gather_idx + r);
+    if (gather_div > 1) idx /= gather_div;
+    uint4* dst = xs + (size_t)r * vec_per_row;
+    if (idx < 0 || idx >= src_rows) {   // a table entry that is no row of the source: reported, the row zero-filled
+      if (lane == 0) report_error(status, DEV_INDEX_OUT_OF_RANGE, KID_DISPATCH, r, idx);
+      for (int v = lane; v < vec_per_row; v += 32) dst[v] = make_uint4(0u, 0u, 0u, 0u);
+      continue;
+    }
+    const uint4* from = src + (size_t)idx * vec_per_row;
+    for (int v0 = 0; v0 < vec_per_row; v0 += 128) {
+      uint4 buf[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int v = v0 + q * 32 + lane;
+        if (v < vec_per_row) buf[q] = __ldg(from + v);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int v = v0 + q * 32 + lane;
+        if (v < vec_per_row) dst[v] = buf[q];
+      }
+    }
+  }
+}
+
+cudaError_t launch_permute_rows(const Shape& s, const void* src, int src_rows, const int32_t* gather_idx,
+                                int gather_div, const int32_t* expert_offsets, void* xs, int32_t* status,
+                                cudaStream_t st) {
+  if (s.T == 0) return cudaSuccess;
+  long long blocks = ((long long)s.T * s.k + 7) / 8;
+  const long long cap = (long long)sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  ProfileScope prof(KID_DISPATCH, st);
+  return launch_pdl(permute_rows_kernel, (unsigned)blocks, 256, 0, st, static_cast<const uint4*>(src),
+                    static_cast<uint4*>(xs), gather_idx, gather_div, expert_offsets, s.E, src_rows, s.d / 8, status);
+}
+
 cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void* xg, cudaStream_t st) {
   if (s.T == 0) return cudaSuccess;
   int blocks = (s.T + 7) / 8;
@@ -237,103 +286,16 @@ cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void
 }
 
 // ---- K5: combine -----------------------------------------------------------------------------
-// One warp per token.  The k slots are visited group by group (ascending group, ascending slot
-// inside a group): the rows of one group are summed first (the pre-reduction that the switch
-// performs per output port), then the group partial joins the token's total; fp32 throughout.
-__device__ __forceinline__ void add_bf16x8(float (&acc)[8], const uint4& raw, float w) {
-  const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&raw);
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const float2 f = __bfloat1622float2(p[q]);
-    acc[2 * q] = fmaf(w, f.x, acc[2 * q]);
-    acc[2 * q + 1] = fmaf(w, f.y, acc[2 * q + 1]);
-  }
-}
-__device__ __forceinline__ uint4 pack_bf16x8(const float (&v)[8]) {
-  uint4 out;
-  __nv_bfloat162* p = reinterpret_cast<__nv_bfloat162*>(&out);
-#pragma unroll
-  for (int q = 0; q < 4; ++q) p[q] = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
-  return out;
-}
-
-__global__ void __launch_bounds__(256) combine_kernel(const uint4* __restrict__ o, uint4* __restrict__ y,
-                                                      uint4* __restrict__ pg, const int32_t* __restrict__ topk_idx,
-                                                      const float* __restrict__ topk_w,
-                                                      const int32_t* __restrict__ pair_row,
-                                                      const int32_t* __restrict__ al,
-                                                      const int32_t* __restrict__ group_offsets, int T, int E, int k,
-                                                      int m, int vec_per_row, int weighted, int n_rows,
-                                                      int32_t* status) {
+// One warp per token; the per-token work is combine_token() (combine.cuh).
+__global__ void __launch_bounds__(256) combine_kernel(const CombineArgs c) {
   grid_dependency_sync();
   __shared__ int s_row[8][32];   // per warp: expert-sorted row of the slot at sorted position p
   __shared__ int s_dst[8][32];   // dispatched row (t, g) of that slot's group
   __shared__ float s_w[8][32];
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const int wpb = blockDim.x >> 5;
-  for (int t = blockIdx.x * wpb + wid; t < T; t += gridDim.x * wpb) {
-    // lane j < k owns slot j; order slots by (group, slot)
-    int my_g = 0x7FFFFFFF, my_row = 0, my_dst = 0;
-    float my_w = 1.f;
-    if (lane < k) {
-      const int e = __ldg(topk_idx + (size_t)t * k + lane);
-      // e < 0: unused slot of a sparse top-k table, sorts behind every real slot and is not read.  An expert
-      // index or a row outside its table (the layout builder reported it and wrote row -1) is skipped the
-      // same way, so no table entry is ever used as an address unchecked.
-      if (e >= 0 && e < E) {
-        const int r = __ldg(pair_row + (size_t)t * k + lane);
-        const int a = __ldg(al + (size_t)(e / m) * T + t);
-        if (r >= 0 && r < n_rows && a >= 0) {
-          my_g = e / m;
-          my_row = r;
-          my_dst = __ldg(group_offsets + my_g) + a;
-          if (weighted) my_w = __ldg(topk_w + (size_t)t * k + lane);
-        } else {
-          report_error(status, DEV_INDEX_OUT_OF_RANGE, KID_COMBINE, t, r);
-        }
-      } else if (e >= E) {
-        report_error(status, DEV_INDEX_OUT_OF_RANGE, KID_COMBINE, t, e);
-      }
-    }
-    const int kv = __popc(__ballot_sync(0xFFFFFFFFu, lane < k && my_g != 0x7FFFFFFF));   // slots in use
-    int my_pos = 0;  // number of slots that come before mine
-    for (int j = 0; j < k; ++j) {
-      const int gj = __shfl_sync(0xFFFFFFFFu, my_g, j);
-      if (gj < my_g || (gj == my_g && j < lane)) ++my_pos;
-    }
-    __syncwarp();
-    if (lane < k) { s_row[wid][my_pos] = my_row; s_dst[wid][my_pos] = my_dst; s_w[wid][my_pos] = my_w; }
-    __syncwarp();
-    for (int v = lane; v < vec_per_row; v += 32) {
-      float total[8], part[8];
-#pragma unroll
-      for (int q = 0; q < 8; ++q) { total[q] = 0.f; part[q] = 0.f; }
-      int prev_dst = -1;
-      for (int s0 = 0; s0 < kv; s0 += 8) {
-        uint4 buf[8];
-#pragma unroll
-        for (int q = 0; q < 8; ++q)   // all loads of the batch are in flight before the first use
-          if (s0 + q < kv) buf[q] = __ldcs(o + (size_t)s_row[wid][s0 + q] * vec_per_row + v);
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          if (s0 + q < kv) {
-            const int dst = s_dst[wid][s0 + q];
-            if (dst != prev_dst && prev_dst >= 0) {   // a group is complete: emit its partial sum
-              if (pg != nullptr) pg[(size_t)prev_dst * vec_per_row + v] = pack_bf16x8(part);
-#pragma unroll
-              for (int c = 0; c < 8; ++c) { total[c] += part[c]; part[c] = 0.f; }
-            }
-            prev_dst = dst;
-            add_bf16x8(part, buf[q], s_w[wid][s0 + q]);
-          }
-        }
-      }
-      if (pg != nullptr && prev_dst >= 0) pg[(size_t)prev_dst * vec_per_row + v] = pack_bf16x8(part);
-#pragma unroll
-      for (int c = 0; c < 8; ++c) total[c] += part[c];
-      y[(size_t)t * vec_per_row + v] = pack_bf16x8(total);
-    }
-  }
+  for (int t = blockIdx.x * wpb + wid; t < c.T; t += gridDim.x * wpb)
+    combine_token<false>(c, t, lane, s_row[wid], s_dst[wid], s_w[wid]);
 }
 
 cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
@@ -343,9 +305,10 @@ cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const
   const int cap = sm_count() * 8;
   if (blocks > cap) blocks = cap;
   ProfileScope prof(KID_COMBINE, st);
-  return launch_pdl(combine_kernel, blocks, 256, 0, st, static_cast<const uint4*>(o), static_cast<uint4*>(y),
-                    static_cast<uint4*>(pg), topk_idx, topk_w, L.pair_row, L.al, L.group_offsets, s.T, s.E, s.k,
-                    s.E / s.G, s.d / 8, (s.flags & 1) ? 1 : 0, s.T * s.k, status);
+  CombineArgs c{static_cast<const uint4*>(o), static_cast<uint4*>(y), static_cast<uint4*>(pg), topk_idx, topk_w,
+                L.pair_row, L.al, L.group_offsets, s.T, s.E, s.k, s.E / s.G, s.d / 8, (s.flags & 1) ? 1 : 0,
+                s.T * s.k, status};
+  return launch_pdl(combine_kernel, blocks, 256, 0, st, c);
 }
 
 // Last step of the layer when Combine ran inside GEMM-2's epilogue: the fp32 token accumulators

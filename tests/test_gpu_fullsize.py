@@ -23,13 +23,32 @@ class Slabs:
         return synth.bf16_bits(self.w[int(e)])
 
 
+def sample_expert_rows(lay, E, rng, per_expert=2, spread=32):
+    """Rows to check expert outputs on: the first and the last row of `spread` experts taken evenly over [0, E)
+    (so a wrong tile decode of any region of the expert range shows), plus the most and the least loaded expert
+    with a few more rows each (first / last / random: both ends of the m-tile range, partial tiles)."""
+    counts = lay["expert_counts"]
+    off = lay["expert_offsets"].astype(np.int64)
+    live = np.nonzero(counts)[0]
+    rows = []
+    for e in np.unique(live[np.linspace(0, live.size - 1, min(spread, live.size)).astype(np.int64)]):
+        rows += [off[e], off[e + 1] - 1][:per_expert]
+    for e in (int(live[np.argmax(counts[live])]), int(live[np.argmin(counts[live])])):
+        lo, hi = int(off[e]), int(off[e + 1])
+        rows += list(range(lo, min(lo + 4, hi))) + list(range(max(hi - 4, lo), hi)) + list(rng.integers(lo, hi, size=4))
+    return np.unique(np.asarray(rows, dtype=np.int64))
+
+
 # C2..C5b: the benchmark configurations; S32 / M16 / L32: three of the paper's own evaluation shapes
 # (Small at top-32 of 64 experts, Medium at top-16, Large at top-32: 2^20 expert rows, element
-# offsets beyond 2^32 in o), 32 groups
-@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C5a", "C5b", "S32", "M16", "L32"])
-def test_fullsize_layer(name):
+# offsets beyond 2^32 in o), 32 groups.  Two more rows run a layer option at full size: Combine inside GEMM-2's
+# epilogue on C4 (its fp32 accumulators outgrow L2 only at this size) and the gate weight applied in Combine on C3.
+@pytest.mark.parametrize("name,flags", [("C2", 0), ("C3", 0), ("C4", 0), ("C5a", 0), ("C5b", 0), ("S32", 0), ("M16", 0),
+                                        ("L32", 0), ("C4", B.MOE_FLAG_COMBINE_IN_EPILOGUE),
+                                        ("C3", B.MOE_FLAG_WEIGHT_IN_COMBINE)])
+def test_fullsize_layer(name, flags):
     cfg = synth.ALL_CONFIGS[name]
-    run = H.Run(cfg)
+    run = H.Run(cfg, flags)
     lay_dev = B.alloc_layout(run.shape)
     run.layer(logits=run.logits, topk_idx=run.idx, topk_w=run.w, layout=lay_dev)
     torch.cuda.synchronize()
@@ -42,40 +61,35 @@ def test_fullsize_layer(name):
     assert lay["n_disp"] <= T * min(k, cfg.G)
     if cfg.G == cfg.E:
         assert lay["n_disp"] == P                     # one expert per group: nothing to de-duplicate
-
-    # expert outputs o (kept in the workspace by moe_layer): sampled rows of sampled experts
-    off = B.moe_workspace_layout(run.shape)
-    o_dev = run.ws[off["o"]: off["o"] + P * cfg.d * 2].view(torch.bfloat16).reshape(P, cfg.d)
-    counts = lay["expert_counts"]
-    live = np.nonzero(counts)[0]
-    rng = np.random.default_rng(1)
-    picks = {int(live[np.argmax(counts[live])]), int(live[np.argmin(counts[live])]), int(rng.choice(live))}
-    rows = []
-    for e in sorted(picks):
-        lo, hi = int(lay["expert_offsets"][e]), int(lay["expert_offsets"][e + 1])
-        take = np.unique(np.concatenate([np.arange(lo, min(lo + 8, hi)), np.arange(max(hi - 8, lo), hi),
-                                         rng.integers(lo, hi, size=8)]))
-        rows.append(take)
-    rows = np.unique(np.concatenate(rows))
     xb = H.bf16_host(run.t["x"])
-    # the fused path feeds GEMM-1 from x; the oracle's dispatched copy holds the same bytes
-    xg = O.dispatch(xb, lay)
     w_gpu = run.host_w()
-    o_ref = O.expert_ffn(xg, lay, w_gpu, Slabs(run.t["w1"]), Slabs(run.t["w3"]), Slabs(run.t["w2"]), rows=rows)
-    o_gpu = O.bf16_to_f64(H.bf16_host(o_dev[torch.from_numpy(rows).cuda()]))
-    H.assert_close_out(o_gpu, o_ref, f"{name} expert rows")
+    in_combine = bool(flags & B.MOE_FLAG_WEIGHT_IN_COMBINE)
 
-    # combine on sampled tokens from the GPU's own o (all k rows of each token)
-    toks = synth.sample_tokens(cfg, 96)
-    need = np.unique(lay["pair_row"].reshape(T, k)[toks].reshape(-1))
-    o_need = O.bf16_to_f64(H.bf16_host(o_dev[torch.from_numpy(need).cuda()]))
-    _, _, y_ref = O.combine(o_need, lay, idx_ref, None, cfg.E, cfg.G, tokens=toks, o_rows=need)
-    y_gpu = O.bf16_to_f64(H.bf16_host(run.y[torch.from_numpy(toks).cuda()]))
-    tol = 2.0 ** -8 * np.abs(y_ref) + 2.0 ** -22 * np.abs(y_ref).max() + 1e-30
-    assert np.all(np.abs(y_gpu - y_ref) <= tol), f"{name} combine"
+    if not flags & B.MOE_FLAG_COMBINE_IN_EPILOGUE:    # (that form never writes o)
+        # expert outputs o (kept in the workspace by moe_layer): two rows of 32 experts spread over the expert range,
+        # more rows of the most and the least loaded expert
+        off = B.moe_workspace_layout(run.shape)
+        o_dev = run.ws[off["o"]: off["o"] + P * cfg.d * 2].view(torch.bfloat16).reshape(P, cfg.d)
+        rows = sample_expert_rows(lay, cfg.E, np.random.default_rng(1))
+        # the fused path feeds GEMM-1 from x; the oracle's dispatched copy holds the same bytes
+        xg = O.dispatch(xb, lay)
+        o_ref = O.expert_ffn(xg, lay, None if in_combine else w_gpu, Slabs(run.t["w1"]), Slabs(run.t["w3"]),
+                             Slabs(run.t["w2"]), rows=rows)
+        o_gpu = O.bf16_to_f64(H.bf16_host(o_dev[torch.from_numpy(rows).cuda()]))
+        H.assert_close_out(o_gpu, o_ref, f"{name} expert rows")
 
-    # whole layer against the dense definition on a few tokens
-    few = synth.sample_tokens(cfg, 96)[:: 96 // 4][:4]
+        # combine on sampled tokens from the GPU's own o (all k rows of each token)
+        toks = synth.sample_tokens(cfg, 96)
+        need = np.unique(lay["pair_row"].reshape(T, k)[toks].reshape(-1))
+        o_need = O.bf16_to_f64(H.bf16_host(o_dev[torch.from_numpy(need).cuda()]))
+        _, _, y_ref = O.combine(o_need, lay, idx_ref, w_gpu if in_combine else None, cfg.E, cfg.G, tokens=toks,
+                                o_rows=need)
+        y_gpu = O.bf16_to_f64(H.bf16_host(run.y[torch.from_numpy(toks).cuda()]))
+        tol = 2.0 ** -8 * np.abs(y_ref) + 2.0 ** -22 * np.abs(y_ref).max() + 1e-30
+        assert np.all(np.abs(y_gpu - y_ref) <= tol), f"{name} combine"
+
+    # whole layer against the dense definition on 16 tokens spread over the batch (first, last and between)
+    few = synth.sample_tokens(cfg, 96)[:: 96 // 16][:16]
     b = run.host_bias()
     _, _, _, y_def = O.layer(xb, run.host_logits(), b, Slabs(run.t["w1"]), Slabs(run.t["w3"]), Slabs(run.t["w2"]),
                              k, cfg.score_fn, tokens=few)
@@ -99,7 +113,7 @@ class QuantSlabs:
         return self.cache[e][self.which]
 
 
-@pytest.mark.parametrize("name", ["C4", "S32"])
+@pytest.mark.parametrize("name", ["C4", "S32", "C5a"])
 def test_fullsize_layer_fp8(name):
     """moe_layer_fp8 at full size: routing and layout in full, quantised operands bit for bit on
     sampled experts, expert outputs on sampled rows and the layer output on sampled tokens."""
@@ -165,7 +179,8 @@ def test_fullsize_single_kernel_ffn_equals_two_kernels(name):
     run.dispatch()
     run.ffn()
     o_two = run.o.clone()
-    for flags in (B.MOE_FLAG_FUSED_FFN, B.MOE_FLAG_FUSED_FFN | B.MOE_FLAG_SM_PARTITION):
+    F, PART, DISP = B.MOE_FLAG_FUSED_FFN, B.MOE_FLAG_SM_PARTITION, B.MOE_FLAG_TRACK_DISPATCH
+    for flags in (F, F | PART, F | DISP):
         fused = H.Run(cfg, flags, inputs=run.t)
         fused.idx, fused.w, fused.lay, fused.xg = run.idx, run.w, run.lay, run.xg
         fused.o.fill_(3.0)
@@ -174,3 +189,27 @@ def test_fullsize_single_kernel_ffn_equals_two_kernels(name):
         assert fused.status()[0] == 0, flags
         assert torch.equal(fused.o[: cfg.P], o_two[: cfg.P]), flags
         del fused
+
+
+@pytest.mark.parametrize("name", ["C3", "C4", "C5a"])
+def test_fullsize_tracker_paced_layer_equals_the_separate_kernels(name):
+    """The whole layer after the layout as one tracker-paced kernel (GEMM-1, GEMM-2 and Combine tasks; with
+    MOE_FLAG_TRACK_DISPATCH also Dispatch tasks; interleaved and with the SM partition) at full size: y must equal
+    the default path (separate GEMM and combine kernels, itself held to the oracle above) bit for bit, and so must
+    the CTA-pair GEMM-1 on the per-expert layout tensors."""
+    cfg = synth.ALL_CONFIGS[name]
+    run = H.Run(cfg)
+    run.layer()
+    torch.cuda.synchronize()
+    assert run.status()[0] == 0
+    y_ref = run.y.clone()
+    F, PART, DISP = B.MOE_FLAG_FUSED_FFN, B.MOE_FLAG_SM_PARTITION, B.MOE_FLAG_TRACK_DISPATCH
+    for flags in (F, F | PART, F | DISP, F | PART | DISP, B.MOE_FLAG_GEMM1_PAIR):
+        other = H.Run(cfg, flags, inputs=run.t)
+        for _ in range(2):                               # the tracker tables are cleared by every call
+            other.y.fill_(5.0)
+            other.layer()
+            torch.cuda.synchronize()
+            assert other.status()[0] == 0, (flags, other.status())
+            assert torch.equal(other.y[: cfg.T], y_ref[: cfg.T]), flags
+        del other

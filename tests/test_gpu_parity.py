@@ -461,10 +461,12 @@ def test_sparse_topk_tables():
 
 @pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
 def test_single_kernel_ffn_with_tile_tracker(cfg):
-    """MOE_FLAG_FUSED_FFN: GEMM-1 and GEMM-2 as one persistent kernel paced by the 128-row tile tracker.  The
-    expert outputs must equal the two-kernel form bit for bit (same operands, same accumulation order per
-    element), in the staged entry point and in the fused layer, twice in a row (the tracker is cleared by every
-    call)."""
+    """MOE_FLAG_FUSED_FFN: the stages after the layout as one persistent kernel paced by the token tracker (tile
+    status counters DAcc / TBCnt1 / TBCnt2 and the per-token output-readiness counter): GEMM-1, GEMM-2, in the layer
+    also the Combine tasks, with MOE_FLAG_TRACK_DISPATCH also the Dispatch tasks, interleaved or with the SM
+    partition.  Expert outputs and y must equal the separate kernels bit for bit (same operands, same accumulation
+    order per element), in the staged entry point and in the fused layer, twice in a row (the tracker is cleared by
+    every call)."""
     if "wcombine" in cfg.name:
         pytest.skip("covered by the default-weight cases")
     run = H.Run(cfg)
@@ -474,7 +476,8 @@ def test_single_kernel_ffn_with_tile_tracker(cfg):
     o_two = run.o.clone()
     run.layer()
     y_two = run.y.clone()
-    for flags in (B.MOE_FLAG_FUSED_FFN, B.MOE_FLAG_FUSED_FFN | B.MOE_FLAG_SM_PARTITION):
+    F, PART, DISP = B.MOE_FLAG_FUSED_FFN, B.MOE_FLAG_SM_PARTITION, B.MOE_FLAG_TRACK_DISPATCH
+    for flags in (F, F | PART, F | DISP, F | PART | DISP):
         _check_single_kernel(cfg, run, flags, o_two, y_two)
 
 
@@ -493,3 +496,22 @@ def _check_single_kernel(cfg, run, flags, o_two, y_two):
         torch.cuda.synchronize()
         assert fused.status()[0] == 0
         assert torch.equal(fused.y[: cfg.T], y_two[: cfg.T])
+
+
+@pytest.mark.parametrize("cfg", SMALL, ids=lambda c: c.name)
+def test_pair_gemm1_on_the_per_expert_layout_tensors(cfg):
+    """MOE_FLAG_GEMM1_PAIR: Dispatch writes one dense row per (token, expert) in expert-sorted order and GEMM-1
+    reads them as TMA tiles on CTA pairs.  Same operands and the same accumulation order per element as the
+    gathering form, so expert outputs and the layer output must equal it bit for bit; the staged path is also held
+    to the oracle."""
+    if "wcombine" in cfg.name:
+        pytest.skip("covered by the default-weight cases")
+    run = H.Run(cfg)
+    run.route()
+    run.dispatch()
+    run.ffn()
+    run.layer()
+    torch.cuda.synchronize()
+    o_ref, y_ref = run.o.clone(), run.y.clone()
+    _check_single_kernel(cfg, run, B.MOE_FLAG_GEMM1_PAIR, o_ref, y_ref)
+    staged(cfg, B.MOE_FLAG_GEMM1_PAIR)

@@ -7,6 +7,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import moe_oracle as O
 from paper_2605_05607_b200 import binding as B
 from paper_2605_05607_b200 import synth
 from tests import helpers as H
@@ -30,6 +31,11 @@ def run_both(cfg):
         assert torch.equal(getattr(lay2, name), getattr(run.lay, name)), name
     assert torch.equal(lay2.disp_token[:n_disp], run.lay.disp_token[:n_disp])
     assert torch.equal(xg2[:n_disp].view(torch.int16), run.xg[:n_disp].view(torch.int16))
+    # and directly against the oracle's layout and dispatched copy of the same routing
+    saved, run.lay, run.xg = (run.lay, run.xg), lay2, xg2
+    lay_ref = H.check_layout(run, run.host_idx())
+    assert np.array_equal(H.bf16_host(xg2)[:n_disp], O.dispatch(H.bf16_host(run.t["x"]), lay_ref))
+    run.lay, run.xg = saved
     return n_disp
 
 
