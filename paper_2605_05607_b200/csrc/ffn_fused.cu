@@ -214,8 +214,12 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
         // Output Readiness table: a token is ready when all topk rows of o are complete
         const int rdy = mine ? ld_acquire(p.nready + my_t) : 0;
         const unsigned ready = __ballot_sync(0xFFFFFFFFu, rdy >= p.k) & pending;
-        for (unsigned rem = ready; rem; rem &= rem - 1)
-          combine_token<true>(p.comb, c * per + (__ffs(rem) - 1), lane, s_row, s_dst, s_w);
+        for (unsigned rem = ready; rem; rem &= rem - 1) {
+          const int t = c * per + (__ffs(rem) - 1);
+          if (p.k <= 2) combine_token<true, 2>(p.comb, t, lane, s_row, s_dst, s_w);
+          else if (p.k <= 4) combine_token<true, 4>(p.comb, t, lane, s_row, s_dst, s_w);
+          else combine_token<true, 8>(p.comb, t, lane, s_row, s_dst, s_w);
+        }
         pending &= ~ready;
         if (pending && !ready) {
           __nanosleep(sleep_ns);

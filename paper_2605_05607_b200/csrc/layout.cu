@@ -183,16 +183,20 @@ cudaError_t launch_layout(const Shape& s, const int32_t* topk_idx, const Layout&
 }
 
 // ---- K3: dispatch ------------------------------------------------------------------------------
-// Token-centric: a warp reads row x[t] once (16-byte vectors) and writes one copy per distinct
-// group the token touches - the single-HBM image of "send once, the switch replicates per port".
+// Token-centric: a warp reads (its part of) row x[t] once (16-byte vectors) and writes one copy per distinct
+// group the token touches - the single-HBM image of "send once, the switch replicates per port".  With few tokens
+// a row is split over `parts` warps (see combine_kernel).
 __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__ x, uint4* __restrict__ xg,
                                                        const int32_t* __restrict__ al,
                                                        const int32_t* __restrict__ group_offsets, int T, int G,
-                                                       int vec_per_row) {
+                                                       int vec_per_row, int parts, int vec_per_part) {
   grid_dependency_sync();
   const int lane = threadIdx.x & 31;
   const int wpb = blockDim.x >> 5;
-  for (int t = blockIdx.x * wpb + (threadIdx.x >> 5); t < T; t += gridDim.x * wpb) {
+  const long long units = (long long)T * parts;
+  for (long long u = (long long)blockIdx.x * wpb + (threadIdx.x >> 5); u < units; u += (long long)gridDim.x * wpb) {
+    const int t = (int)(u / parts), part = (int)(u % parts);
+    const int v_lo = part * vec_per_part, v_hi = min(vec_per_row, v_lo + vec_per_part);
     const uint4* src = x + (size_t)t * vec_per_row;
     for (int g0 = 0; g0 < G; g0 += 32) {
       const int g = g0 + lane;
@@ -203,12 +207,12 @@ __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__
       }
       unsigned live = __ballot_sync(0xFFFFFFFFu, dst_row >= 0);
       if (!live) continue;
-      for (int v0 = 0; v0 < vec_per_row; v0 += 128) {
+      for (int v0 = v_lo; v0 < v_hi; v0 += 128) {
         uint4 buf[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
           const int v = v0 + q * 32 + lane;
-          if (v < vec_per_row) buf[q] = __ldcs(src + v);
+          if (v < v_hi) buf[q] = __ldcs(src + v);
         }
         for (unsigned rem = live; rem; rem &= rem - 1) {
           const int row = __shfl_sync(0xFFFFFFFFu, dst_row, __ffs(rem) - 1);
@@ -216,12 +220,27 @@ __global__ void __launch_bounds__(256) dispatch_kernel(const uint4* __restrict__
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
             const int v = v0 + q * 32 + lane;
-            if (v < vec_per_row) __stcs(dst + v, buf[q]);
+            if (v < v_hi) __stcs(dst + v, buf[q]);
           }
         }
       }
     }
   }
+}
+
+static int row_parts(int T, int vec_per_row);
+
+cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void* xg, cudaStream_t st) {
+  if (s.T == 0) return cudaSuccess;
+  const int vec = s.d / 8;
+  const int parts = row_parts(s.T, vec);
+  const int vec_per_part = ((vec + parts - 1) / parts + 127) & ~127;   // whole 128-vector steps per part
+  long long blocks = ((long long)s.T * parts + 7) / 8;
+  const long long cap = (long long)sm_count() * 8;
+  if (blocks > cap) blocks = cap;
+  ProfileScope prof(KID_DISPATCH, st);
+  return launch_pdl(dispatch_kernel, (unsigned)blocks, 256, 0, st, static_cast<const uint4*>(x), static_cast<uint4*>(xg),
+                    L.al, L.group_offsets, s.T, s.G, vec, parts, vec_per_part);
 }
 
 // ---- K3b: dispatch into the per-expert layout tensors ----------------------------------------------
@@ -275,40 +294,49 @@ cudaError_t launch_permute_rows(const Shape& s, const void* src, int src_rows, c
                     static_cast<uint4*>(xs), gather_idx, gather_div, expert_offsets, s.E, src_rows, s.d / 8, status);
 }
 
-cudaError_t launch_dispatch(const Shape& s, const void* x, const Layout& L, void* xg, cudaStream_t st) {
-  if (s.T == 0) return cudaSuccess;
-  int blocks = (s.T + 7) / 8;
-  const int cap = sm_count() * 8;
-  if (blocks > cap) blocks = cap;
-  ProfileScope prof(KID_DISPATCH, st);
-  return launch_pdl(dispatch_kernel, blocks, 256, 0, st, static_cast<const uint4*>(x), static_cast<uint4*>(xg), L.al,
-                    L.group_offsets, s.T, s.G, s.d / 8);
-}
-
 // ---- K5: combine -----------------------------------------------------------------------------
-// One warp per token; the per-token work is combine_token() (combine.cuh).
-__global__ void __launch_bounds__(256) combine_kernel(const CombineArgs c) {
+// One warp per (token, column part); the per-token work is combine_token() (combine.cuh).  With few tokens a row
+// is split over `parts` warps so that enough loads are in flight to reach the memory bandwidth (one warp per token
+// leaves a 4096-token batch at a third of it).
+template <int BATCH>
+__global__ void __launch_bounds__(256, 3) combine_kernel(const CombineArgs c, int parts, int vec_per_part) {
   grid_dependency_sync();
   __shared__ int s_row[8][32];   // per warp: expert-sorted row of the slot at sorted position p
   __shared__ int s_dst[8][32];   // dispatched row (t, g) of that slot's group
   __shared__ float s_w[8][32];
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const int wpb = blockDim.x >> 5;
-  for (int t = blockIdx.x * wpb + wid; t < c.T; t += gridDim.x * wpb)
-    combine_token<false>(c, t, lane, s_row[wid], s_dst[wid], s_w[wid]);
+  const long long units = (long long)c.T * parts;
+  for (long long u = (long long)blockIdx.x * wpb + wid; u < units; u += (long long)gridDim.x * wpb) {
+    const int t = (int)(u / parts), part = (int)(u % parts);
+    combine_token<false, BATCH>(c, t, lane, s_row[wid], s_dst[wid], s_w[wid], part * vec_per_part,
+                                (part + 1) * vec_per_part);
+  }
+}
+
+// parts of a row so that about 32 warps per SM exist even for small batches (at most 8, at least 4 vectors per lane)
+static int row_parts(int T, int vec_per_row) {
+  int parts = 1;
+  while (parts < 8 && (long long)T * parts < 32ll * sm_count() * 2 && vec_per_row / (parts * 2) >= 128) parts *= 2;
+  return parts;
 }
 
 cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
                            const float* topk_w, void* pg, void* y, int32_t* status, cudaStream_t st) {
   if (s.T == 0) return cudaSuccess;
-  int blocks = (s.T + 7) / 8;
-  const int cap = sm_count() * 8;
+  const int vec = s.d / 8;
+  const int parts = row_parts(s.T, vec);
+  const int vec_per_part = ((vec + parts - 1) / parts + 31) & ~31;   // whole warp-strides per part
+  long long blocks = ((long long)s.T * parts + 7) / 8;
+  const long long cap = (long long)sm_count() * 8;
   if (blocks > cap) blocks = cap;
   ProfileScope prof(KID_COMBINE, st);
   CombineArgs c{static_cast<const uint4*>(o), static_cast<uint4*>(y), static_cast<uint4*>(pg), topk_idx, topk_w,
-                L.pair_row, L.al, L.group_offsets, s.T, s.E, s.k, s.E / s.G, s.d / 8, (s.flags & 1) ? 1 : 0,
+                L.pair_row, L.al, L.group_offsets, s.T, s.E, s.k, s.E / s.G, vec, (s.flags & 1) ? 1 : 0,
                 s.T * s.k, status};
-  return launch_pdl(combine_kernel, blocks, 256, 0, st, c);
+  if (s.k <= 2) return launch_pdl(combine_kernel<2>, (unsigned)blocks, 256, 0, st, c, parts, vec_per_part);
+  if (s.k <= 4) return launch_pdl(combine_kernel<4>, (unsigned)blocks, 256, 0, st, c, parts, vec_per_part);
+  return launch_pdl(combine_kernel<8>, (unsigned)blocks, 256, 0, st, c, parts, vec_per_part);
 }
 
 // Last step of the layer when Combine ran inside GEMM-2's epilogue: the fp32 token accumulators
