@@ -40,7 +40,9 @@ Pins: every function below is pinned by tests that do not re-type its formula:
 pure-Python brute force over all (token, expert) / (token, group) pairs, a
 hand-worked layout example, closed forms (k = 1, equal keys, two-key softmax =
 logistic), invariants, the dense-MLP special case, and the paper's printed
-340 % / "nearly 50 %" traffic figures for the distinct-group counter.
+340 % / "nearly 50 %" traffic figures for the distinct-group counter; the backward functions
+by central finite differences of the (pinned) forward and by fp64 automatic differentiation of the
+dense single-expert case; the packet model by the paper's printed 80 % -> 69 %.
 """
 from __future__ import annotations
 
@@ -189,18 +191,20 @@ def dispatch(x_bits: np.ndarray, lay: Dict[str, np.ndarray]) -> np.ndarray:
 
 
 # --------------------------------------------------------------------------- experts
-def expert_ffn_rows(a: np.ndarray, w1_bits: np.ndarray, w3_bits: np.ndarray,
-                    w2_bits: np.ndarray) -> np.ndarray:
-    """One expert applied to rows ``a`` (float64 [n, d]):
-    GEMM-1  a1 = a W1, a3 = a W3 ;  h = silu(a1) * a3 ;  GEMM-2  o = h W2.
-    All in fp64, no intermediate rounding."""
-    w1 = bf16_to_f64(w1_bits)
-    w3 = bf16_to_f64(w3_bits)
-    w2 = bf16_to_f64(w2_bits)
+def expert_ffn_rows_f64(a: np.ndarray, w1: np.ndarray, w3: np.ndarray, w2: np.ndarray) -> np.ndarray:
+    """One expert with float64 weights applied to rows ``a`` (float64 [n, d]):
+    GEMM-1  a1 = a W1, a3 = a W3 ;  h = silu(a1) * a3 ;  GEMM-2  o = h W2."""
     a1 = a @ w1
     a3 = a @ w3
     h = a1 / (1.0 + np.exp(-a1)) * a3
     return h @ w2
+
+
+def expert_ffn_rows(a: np.ndarray, w1_bits: np.ndarray, w3_bits: np.ndarray,
+                    w2_bits: np.ndarray) -> np.ndarray:
+    """One expert applied to rows ``a`` (float64 [n, d]), weights given as bf16 bits.
+    All in fp64, no intermediate rounding."""
+    return expert_ffn_rows_f64(a, bf16_to_f64(w1_bits), bf16_to_f64(w3_bits), bf16_to_f64(w2_bits))
 
 
 def expert_ffn(xg_bits: np.ndarray, lay: Dict[str, np.ndarray], topk_w: Optional[np.ndarray],
@@ -287,6 +291,51 @@ def layer(x_bits: np.ndarray, logits: np.ndarray, bias: Optional[np.ndarray],
         o = expert_ffn_rows(a, w1_bits[e], w3_bits[e], w2_bits[e])
         y[hit_t] += w[toks[hit_t], hit_j][:, None] * o
     return toks, sel_idx, w[toks], y
+
+
+# --------------------------------------------------------------------------- backward
+def expert_ffn_rows_backward_f64(a: np.ndarray, w1: np.ndarray, w3: np.ndarray, w2: np.ndarray, do: np.ndarray):
+    """Gradients of  sum(do * o),  o = (silu(a W1) * (a W3)) W2,  with respect to a, W1, W3, W2 (the chain rule
+    written out, fp64).  ``do`` is float64 [n, d].  Returns (da, dW1, dW3, dW2)."""
+    a1 = a @ w1
+    a3 = a @ w3
+    s = 1.0 / (1.0 + np.exp(-a1))
+    silu = a1 * s
+    h = silu * a3
+    dh = do @ w2.T
+    da3 = dh * silu
+    da1 = dh * a3 * (s * (1.0 + a1 * (1.0 - s)))     # d silu(u) / du = s (1 + u (1 - s))
+    da = da1 @ w1.T + da3 @ w3.T
+    return da, a.T @ da1, a.T @ da3, h.T @ do
+
+
+def layer_backward(x_bits: np.ndarray, topk_idx: np.ndarray, topk_w: np.ndarray, w1_bits, w3_bits, w2_bits,
+                   dy: np.ndarray, experts: Optional[Sequence[int]] = None):
+    """Backward pass of the layer for FIXED routing (Sec. VI-A evaluates training, forward + backward): with
+    y[t] = sum_j w[t, j] * FFN_{idx[t, j]}(x[t])  and the expert indices and gate weights held constant,
+    the gradients of  L = sum(dy * y)  are
+        dx[t]  = sum_j  w[t, j] * dFFN/da (x[t]) applied to dy[t]
+        dW*[e] = sum over the pairs (t, j) with idx[t, j] = e  of  w[t, j] * (their expert-level gradient).
+    ``dy`` float64 [T, d]; ``topk_w`` [T, k].  With ``experts`` only those experts' weight gradients are formed
+    (dx is then omitted).  Returns (dx [T, d] or None, {e: (dW1, dW3, dW2)}), all float64."""
+    idx = np.asarray(topk_idx, dtype=np.int64)
+    w = np.asarray(topk_w, dtype=np.float64)
+    T = x_bits.shape[0]
+    dx = np.zeros((T, x_bits.shape[1]), dtype=np.float64) if experts is None else None
+    grads = {}
+    for e in (np.unique(idx) if experts is None else experts):
+        hit_t, hit_j = np.nonzero(idx == e)
+        w1, w3, w2 = bf16_to_f64(w1_bits[e]), bf16_to_f64(w3_bits[e]), bf16_to_f64(w2_bits[e])
+        if hit_t.size == 0:
+            grads[int(e)] = (np.zeros_like(w1), np.zeros_like(w3), np.zeros_like(w2))
+            continue
+        a = bf16_to_f64(x_bits[hit_t])
+        do = w[hit_t, hit_j][:, None] * np.asarray(dy, dtype=np.float64)[hit_t]
+        da, g1, g3, g2 = expert_ffn_rows_backward_f64(a, w1, w3, w2, do)
+        if dx is not None:
+            np.add.at(dx, hit_t, da)
+        grads[int(e)] = (g1, g3, g2)
+    return dx, grads
 
 
 # --------------------------------------------------------------------------- traffic counters

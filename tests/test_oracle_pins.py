@@ -489,3 +489,93 @@ def test_payload_efficiency_reproduces_the_papers_printed_pair(golden_dir):
     for n in range(1, 33):
         a, b = O.payload_efficiency(640, n), O.payload_efficiency(640, n - 1)
         assert a["explicit"] < b["explicit"] and a["dynamic"] <= b["dynamic"]
+
+
+# ------------------------------------------------------------------------------------------------ backward
+def _rand_expert(rng, n, d, f):
+    return (rng.standard_normal((n, d)), rng.standard_normal((d, f)) / np.sqrt(d),
+            rng.standard_normal((d, f)) / np.sqrt(d), rng.standard_normal((f, d)) / np.sqrt(f))
+
+
+def test_expert_backward_against_central_finite_differences():
+    """Every entry of da, dW1, dW3, dW2 of a tiny expert against a central difference of the forward (which has its
+    own pins): a dropped term, a wrong sign in the derivative of silu or a transposed operand fails it."""
+    rng = np.random.default_rng(3)
+    a, w1, w3, w2 = _rand_expert(rng, 3, 5, 4)
+    do = rng.standard_normal((3, 5))
+    da, g1, g3, g2 = O.expert_ffn_rows_backward_f64(a, w1, w3, w2, do)
+    loss = lambda a_, w1_, w3_, w2_: float((do * O.expert_ffn_rows_f64(a_, w1_, w3_, w2_)).sum())
+    eps = 1e-6
+    for arr, grad, pos in ((a, da, 0), (w1, g1, 1), (w3, g3, 2), (w2, g2, 3)):
+        num = np.zeros_like(arr)
+        for i in np.ndindex(arr.shape):
+            args = [a, w1, w3, w2]
+            hi, lo = arr.copy(), arr.copy()
+            hi[i] += eps
+            lo[i] -= eps
+            args[pos] = hi
+            up = loss(*args)
+            args[pos] = lo
+            num[i] = (up - loss(*args)) / (2 * eps)
+        assert np.abs(num - grad).max() <= 1e-7 * max(1.0, np.abs(grad).max()), pos
+
+
+def test_expert_backward_against_fp64_autograd():
+    """The dense special case (one expert, every row) against torch's fp64 automatic differentiation."""
+    rng = np.random.default_rng(4)
+    a, w1, w3, w2 = _rand_expert(rng, 7, 12, 9)
+    do = rng.standard_normal((7, 12))
+    ta, t1, t3, t2 = (torch.tensor(v, dtype=torch.float64, requires_grad=True) for v in (a, w1, w3, w2))
+    out = (torch.nn.functional.silu(ta @ t1) * (ta @ t3)) @ t2
+    (out * torch.tensor(do)).sum().backward()
+    got = O.expert_ffn_rows_backward_f64(a, w1, w3, w2, do)
+    for g, t in zip(got, (ta, t1, t3, t2)):
+        assert np.abs(g - t.grad.numpy()).max() <= 1e-12 * max(1.0, np.abs(g).max())
+
+
+def test_layer_backward_is_the_routed_sum_of_expert_gradients():
+    """layer_backward on a small routed layer: dx and the weight gradients against a finite difference of the
+    oracle's own forward with the routing held fixed (tokens perturbed one coordinate at a time through the dense
+    definition), plus the structural facts: experts nobody selected get zero gradients, the result is linear in
+    dy, and the gate weight multiplies the expert-level gradient."""
+    rng = np.random.default_rng(5)
+    T, d, f, E, k = 6, 8, 8, 4, 2
+    xb = O.f64_to_bf16_bits(rng.standard_normal((T, d)))
+    w1b, w3b, w2b = (O.f64_to_bf16_bits(rng.standard_normal(s) * 0.4) for s in ((E, d, f), (E, d, f), (E, f, d)))
+    idx = np.array([[0, 1], [1, 3], [3, 0], [0, 3], [1, 0], [3, 1]], dtype=np.int32)       # expert 2 unused
+    w = rng.uniform(0.2, 0.8, size=(T, k))
+    dy = rng.standard_normal((T, d))
+    dx, grads = O.layer_backward(xb, idx, w, w1b, w3b, w2b, dy)
+
+    def forward(x64):       # dense definition with the routing fixed, float64 tokens
+        y = np.zeros((T, d))
+        for t in range(T):
+            for j in range(k):
+                e = idx[t, j]
+                y[t] += w[t, j] * O.expert_ffn_rows_f64(x64[t:t + 1], O.bf16_to_f64(w1b[e]), O.bf16_to_f64(w3b[e]),
+                                                        O.bf16_to_f64(w2b[e]))[0]
+        return y
+
+    x64 = O.bf16_to_f64(xb)
+    eps = 1e-6
+    num = np.zeros_like(x64)
+    for i in np.ndindex(x64.shape):
+        hi, lo = x64.copy(), x64.copy()
+        hi[i] += eps
+        lo[i] -= eps
+        num[i] = ((dy * forward(hi)).sum() - (dy * forward(lo)).sum()) / (2 * eps)
+    assert np.abs(num - dx).max() <= 1e-6 * max(1.0, np.abs(dx).max())
+    # expert 2 was never selected: no entry in the routed result, zeros when asked for explicitly
+    assert 2 not in grads
+    _, only2 = O.layer_backward(xb, idx, w, w1b, w3b, w2b, dy, experts=[2])
+    assert all(not g.any() for g in only2[2])
+    # weight gradient of expert 3 = sum over its pairs of w * (expert-level gradient of that row)
+    g1 = np.zeros((d, f))
+    for t, j in zip(*np.nonzero(idx == 3)):
+        _, r1, _, _ = O.expert_ffn_rows_backward_f64(x64[t:t + 1], O.bf16_to_f64(w1b[3]), O.bf16_to_f64(w3b[3]),
+                                                     O.bf16_to_f64(w2b[3]), dy[t:t + 1])
+        g1 += w[t, j] * r1
+    assert np.abs(g1 - grads[3][0]).max() <= 1e-12 * max(1.0, np.abs(g1).max())
+    # linear in dy
+    dx2, grads2 = O.layer_backward(xb, idx, w, w1b, w3b, w2b, 2.0 * dy)
+    assert np.array_equal(dx2, 2.0 * dx) and np.array_equal(grads2[0][2], 2.0 * grads[0][2])
