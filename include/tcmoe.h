@@ -212,6 +212,26 @@ int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, co
                    const void* w1, const void* w3, const void* w2, void* y_dev, void* y_host,
                    void* ws, size_t ws_bytes, void* stream);
 
+/* ---- backward pass ----------------------------------------------------------------------------------
+ * Sec. VI-A evaluates training, forward + backward, of the layer of Sec. II-A.  For FIXED routing (expert indices
+ * and gate weights as the forward produced them, held constant: the gate network's own gradient is not part of
+ * this call), with dy = dL/dy:
+ *     dx[t]  = sum_j w[t,j] * dFFN_e/da (x[t]) applied to dy[t]          [T, d] bf16
+ *     dw1[e] = Xs_e^T dA1_e,  dw3[e] = Xs_e^T dA3_e,  dw2[e] = H_e^T dO_e   [E, d, f], [E, d, f], [E, f, d] bf16
+ * where Xs_e / H_e / dO_e / dA*_e are the rows of expert e (dO = w * dy, dH = dO W2^T, dA1 = dH * a3 * silu'(a1),
+ * dA3 = dH * silu(a1), a1 = x W1, a3 = x W3 recomputed).  bf16 operands, fp32 accumulation, intermediates rounded
+ * to bf16.  Weight gradients are written in full (zeros for experts no token selected).
+ *   x, dy       [T, d] bf16
+ *   topk_idx, topk_w, layout   as written by moe_layer / moe_route + moe_dispatch for the same x
+ *   w1, w3, w2  the forward weights, read in place (transposed operands are read K-major, nothing is repacked)
+ *   ws          moe_backward_workspace_bytes(shape) bytes, 128-byte aligned, status block at its start (zero it
+ *               once or call moe_status_reset; read with moe_status)
+ * shape->flags: 0 or MOE_FLAG_SPARSE_TOPK. */
+int moe_backward_workspace_bytes(const moe_shape_t* shape, size_t* bytes);
+int moe_layer_backward(const moe_shape_t* shape, const void* x, const void* dy, const int32_t* topk_idx,
+                       const float* topk_w, const moe_layout_t* layout, const void* w1, const void* w3, const void* w2,
+                       void* dx, void* dw1, void* dw3, void* dw2, void* ws, size_t ws_bytes, void* stream);
+
 /* ---- FP8 form of the expert FFN --------------------------------------------------------------
  * Sec. V-A evaluates the DeepSeek-V3 experts with FP8 GEMM kernels and gives no recipe; this
  * library's reading: E4M3 elements (largest finite value 448, round to nearest even, saturating),
@@ -290,7 +310,8 @@ int moe_workspace_layout(const moe_shape_t* shape, size_t out[4]);
 
 /* Kernel ids for moe_profile_enable (also the `where` slot of moe_status). */
 enum { MOE_KERNEL_TOPK = 1, MOE_KERNEL_MASKS = 2, MOE_KERNEL_FILL = 3, MOE_KERNEL_DISPATCH = 4,
-       MOE_KERNEL_GEMM1 = 5, MOE_KERNEL_GEMM2 = 6, MOE_KERNEL_COMBINE = 7, MOE_KERNEL_GATE = 8 };
+       MOE_KERNEL_GEMM1 = 5, MOE_KERNEL_GEMM2 = 6, MOE_KERNEL_COMBINE = 7, MOE_KERNEL_GATE = 8,
+       MOE_KERNEL_WGRAD = 10, MOE_KERNEL_BWD_GATHER = 11 };
 
 /* Per-kernel timing hook for benchmarks (host-side state, one record per process, guarded by a
  * mutex so that launches from several host threads are safe; not part of the method).  After moe_profile_enable(id) every launch of that kernel by any entry point is

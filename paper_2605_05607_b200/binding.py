@@ -44,7 +44,7 @@ EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "m
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",
            "moe_profile_enable", "moe_profile_read", "moe_dispatch_noalloc", "moe_quantize_rows",
            "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8", "moe_layer_fp8_host", "moe_selftest_wait_timeout", "moe_traffic_stats", "moe_ep_pack", "moe_ep_finish",
-           "moe_payload_efficiency")
+           "moe_payload_efficiency", "moe_backward_workspace_bytes", "moe_layer_backward")
 
 
 class MoEShape(ctypes.Structure):
@@ -97,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.moe_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint64, vp]
         L.moe_traffic_stats.argtypes = [shp, lay, ctypes.POINTER(ctypes.c_double), vp]
         L.moe_payload_efficiency.argtypes = [i64, ctypes.c_int32, ctypes.POINTER(ctypes.c_double)]
+        L.moe_backward_workspace_bytes.argtypes = [shp, ctypes.POINTER(sz)]
+        L.moe_layer_backward.argtypes = [shp, vp, vp, vp, vp, lay, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         L.moe_ep_pack.argtypes = [shp, vp, vp, lay, vp, vp, vp]
         L.moe_ep_finish.argtypes = [shp, vp, lay, vp, vp]
         L.moe_profile_enable.argtypes = [ctypes.c_int]
@@ -283,6 +285,21 @@ def moe_payload_efficiency(transfer_bytes: int, n_targets: int) -> dict:
     return dict(zip(("data_flits", "ideal", "explicit", "dynamic"), list(out)))
 
 
+def moe_backward_workspace_bytes(shape: MoEShape) -> int:
+    out = ctypes.c_size_t(0)
+    _check("moe_backward_workspace_bytes", lib().moe_backward_workspace_bytes(ctypes.byref(shape), ctypes.byref(out)))
+    return out.value
+
+
+def moe_layer_backward(shape, x, dy, topk_idx, topk_w, layout: Layout, w1, w3, w2, dx, dw1, dw3, dw2, ws,
+                       stream=None) -> None:
+    c = layout.c()
+    _check("moe_layer_backward", lib().moe_layer_backward(ctypes.byref(shape), _ptr(x), _ptr(dy), _ptr(topk_idx),
+                                                          _ptr(topk_w), ctypes.byref(c), _ptr(w1), _ptr(w3), _ptr(w2),
+                                                          _ptr(dx), _ptr(dw1), _ptr(dw3), _ptr(dw2), _ptr(ws),
+                                                          ws.numel(), _stream(stream)))
+
+
 def moe_selftest_wait_timeout(ws, limit_ns: int, stream=None) -> None:
     _check("moe_selftest_wait_timeout", lib().moe_selftest_wait_timeout(_ptr(ws), limit_ns, _stream(stream)))
 
@@ -310,7 +327,8 @@ def moe_layer_host(shape, x_host, x_dev, w_gate, logit_bias, w1, w3, w2, y_dev, 
                                                   _ptr(y_dev), _ptr(y_host), _ptr(ws), ws.numel(), _stream(stream)))
 
 
-KERNEL_IDS = {"topk": 1, "masks": 2, "fill": 3, "dispatch": 4, "gemm1": 5, "gemm2": 6, "combine": 7, "gate": 8}
+KERNEL_IDS = {"topk": 1, "masks": 2, "fill": 3, "dispatch": 4, "gemm1": 5, "gemm2": 6, "combine": 7, "gate": 8,
+              "wgrad": 10, "bwd_gather": 11}
 
 
 def moe_profile_enable(kernel_id: int) -> None:

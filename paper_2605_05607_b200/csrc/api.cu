@@ -290,7 +290,7 @@ int moe_selftest_wait_timeout(void* ws, uint64_t limit_ns, void* stream) {
 }
 
 int moe_profile_enable(int kernel_id) {
-  if (kernel_id < 0 || kernel_id > 8) return MOE_ERR_INVALID_ARG;
+  if (kernel_id < 0 || kernel_id > 11) return MOE_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_profile_mutex);
   g_profile_id.store(kernel_id, std::memory_order_relaxed);
   g_profile_n = 0;
@@ -448,6 +448,94 @@ int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t*
   TCMOE_CUDA(launch_tile_prefix(to_shape(*shape), layout->expert_counts, at<int32_t>(ws, p.mt_prefix),
                                 at<int32_t>(ws, p.mp_prefix), static_cast<cudaStream_t>(stream)));
   TCMOE_CUDA(launch_expert_ffn(to_shape(*shape), a, static_cast<cudaStream_t>(stream)));
+  return MOE_OK;
+}
+
+namespace tcmoe {
+namespace {
+// Regions of the backward workspace, in order, each on a 1 KiB boundary.
+struct BwdPlan {
+  size_t status, poff, mt_prefix, mp_prefix, pair_prow, xs, dos, dh, h, da1, da3, dxs, total;
+};
+BwdPlan bwd_plan(const moe_shape_t& s) {
+  BwdPlan p{};
+  const size_t E = (size_t)s.E, P = (size_t)s.T * s.k;
+  const size_t R = bwd_row_capacity(to_shape(s));
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t at = off;
+    off = round_up(off + bytes, ALIGN);
+    return at;
+  };
+  p.status = take(64);
+  p.poff = take((E + 1) * 4);
+  p.mt_prefix = take((E + 1) * 4);
+  p.mp_prefix = take((E + 1) * 4);
+  p.pair_prow = take(P * 4);
+  p.xs = take(R * (size_t)s.d * 2);
+  p.dos = take(R * (size_t)s.d * 2);
+  p.dh = take(R * (size_t)s.f * 2);
+  p.h = take(R * (size_t)s.f * 2);
+  p.da1 = take(R * (size_t)s.f * 2);
+  p.da3 = take(R * (size_t)s.f * 2);
+  p.dxs = take(R * (size_t)s.d * 2);
+  p.total = off;
+  return p;
+}
+}  // namespace
+}  // namespace tcmoe
+
+int moe_backward_workspace_bytes(const moe_shape_t* shape, size_t* bytes) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (bytes == nullptr) return MOE_ERR_INVALID_ARG;
+  *bytes = bwd_plan(*shape).total;
+  return MOE_OK;
+}
+
+int moe_layer_backward(const moe_shape_t* shape, const void* x, const void* dy, const int32_t* topk_idx,
+                       const float* topk_w, const moe_layout_t* layout, const void* w1, const void* w3, const void* w2,
+                       void* dx, void* dw1, void* dw3, void* dw2, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (shape->flags & ~MOE_FLAG_SPARSE_TOPK) return MOE_ERR_INVALID_ARG;   // the forward's kernel-form flags do not apply
+  if (x == nullptr || dy == nullptr || topk_idx == nullptr || topk_w == nullptr || w1 == nullptr || w3 == nullptr ||
+      w2 == nullptr || dx == nullptr || dw1 == nullptr || dw3 == nullptr || dw2 == nullptr || ws == nullptr)
+    return MOE_ERR_INVALID_ARG;
+  if ((rc = check_layout(layout)) != MOE_OK) return rc;
+  if (!aligned(x, 128) || !aligned(dy, 128) || !aligned(w1, 128) || !aligned(w3, 128) || !aligned(w2, 128) ||
+      !aligned(dx, 128) || !aligned(dw1, 128) || !aligned(dw3, 128) || !aligned(dw2, 128) || !aligned(ws, 128) ||
+      !aligned(topk_idx, 16) || !aligned(topk_w, 16))
+    return MOE_ERR_MISALIGNED;
+  const BwdPlan p = bwd_plan(*shape);
+  if (ws_bytes < p.total) return MOE_ERR_WORKSPACE_TOO_SMALL;
+  if (!have_device()) return MOE_ERR_CUDA;
+  BwdArgs a{};
+  a.x = x;
+  a.dy = dy;
+  a.topk_idx = topk_idx;
+  a.topk_w = topk_w;
+  a.L = to_layout(*layout);
+  a.w1 = w1;
+  a.w3 = w3;
+  a.w2 = w2;
+  a.dx = dx;
+  a.dw1 = dw1;
+  a.dw3 = dw3;
+  a.dw2 = dw2;
+  a.poff = at<int32_t>(ws, p.poff);
+  a.mt_prefix = at<int32_t>(ws, p.mt_prefix);
+  a.mp_prefix = at<int32_t>(ws, p.mp_prefix);
+  a.pair_prow = at<int32_t>(ws, p.pair_prow);
+  a.xs = at<void>(ws, p.xs);
+  a.dos = at<void>(ws, p.dos);
+  a.dh = at<void>(ws, p.dh);
+  a.h = at<void>(ws, p.h);
+  a.da1 = at<void>(ws, p.da1);
+  a.da3 = at<void>(ws, p.da3);
+  a.dxs = at<void>(ws, p.dxs);
+  a.status = at<int32_t>(ws, p.status);
+  TCMOE_CUDA(launch_layer_backward(to_shape(*shape), a, static_cast<cudaStream_t>(stream)));
   return MOE_OK;
 }
 

@@ -9,7 +9,7 @@ namespace tcmoe {
 // ---- status block at the start of the workspace (16 x int32) --------------------------------
 enum StatusSlot { ST_CODE = 0, ST_WHERE = 1, ST_DETAIL = 2, ST_AUX = 3, ST_ABORT = 4, ST_WARN = 5 };
 enum KernelId { KID_TOPK = 1, KID_MASKS = 2, KID_FILL = 3, KID_DISPATCH = 4, KID_GEMM1 = 5, KID_GEMM2 = 6,
-                KID_COMBINE = 7, KID_GATE = 8 };
+                KID_COMBINE = 7, KID_GATE = 8, KID_SELFTEST = 9, KID_WGRAD = 10, KID_BWD = 11 };
 constexpr int DEV_TIMEOUT = 1;
 constexpr int DEV_INDEX_OUT_OF_RANGE = 2;
 constexpr int WARN_NONFINITE_LOGIT = 1;
@@ -104,6 +104,23 @@ cudaError_t launch_permute_rows(const Shape& s, const void* src, int src_rows, c
 cudaError_t launch_round_rows(const Shape& s, const float* acc, void* y, cudaStream_t st);
 cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
                            const float* topk_w, void* pg, void* y, int32_t* status, cudaStream_t st);
+cudaError_t launch_combine_rows(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
+                                const float* topk_w, void* pg, void* y, int n_rows, int32_t* status, cudaStream_t st);
+// bwd.cu: backward pass of the layer for fixed routing
+struct BwdArgs {
+  const void *x, *dy;               // [T, d] bf16
+  const int32_t* topk_idx;          // [T, k]
+  const float* topk_w;              // [T, k]
+  Layout L;                         // the forward layout
+  const void *w1, *w3, *w2;         // forward weights
+  void *dx, *dw1, *dw3, *dw2;       // outputs
+  // scratch (padded row space: bwd_row_capacity() rows each)
+  int32_t *poff, *mt_prefix, *mp_prefix, *pair_prow;
+  void *xs, *dos, *dh, *h, *da1, *da3, *dxs;
+  int32_t* status;
+};
+size_t bwd_row_capacity(const Shape& s);
+cudaError_t launch_layer_backward(const Shape& s, const BwdArgs& a, cudaStream_t st);
 // ffn.cu
 struct FfnArgs {
   const void* a_src;          // GEMM-1 activations: xg (gather_div = 1) or x (gather_div = k)

@@ -5,18 +5,17 @@
 #include <atomic>
 
 namespace tcmoe {
+namespace ffn {
 
-namespace {
-
-ffn::EncodeTiledFn encode_fn() {
-  static std::atomic<ffn::EncodeTiledFn> cached{nullptr};   // looked up once; a second lookup gives the same address
-  ffn::EncodeTiledFn fn = cached.load(std::memory_order_acquire);
+EncodeTiledFn encode_fn() {
+  static std::atomic<EncodeTiledFn> cached{nullptr};   // looked up once; a second lookup gives the same address
+  EncodeTiledFn fn = cached.load(std::memory_order_acquire);
   if (fn == nullptr) {
     void* sym = nullptr;
     cudaDriverEntryPointQueryResult q;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
         q == cudaDriverEntryPointSuccess) {
-      fn = reinterpret_cast<ffn::EncodeTiledFn>(sym);
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
       cached.store(fn, std::memory_order_release);
     }
   }
@@ -25,11 +24,11 @@ ffn::EncodeTiledFn encode_fn() {
 
 // bf16 weights [E, K, N] row-major: box = 64 (N) x 64 (K) x 1, 128-byte swizzle, zero fill
 bool make_weight_map(CUtensorMap* map, const void* base, int E, int K, int N) {
-  ffn::EncodeTiledFn fn = encode_fn();
+  EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)K, (cuuint64_t)E};
   cuuint64_t strides[2] = {(cuuint64_t)N * 2, (cuuint64_t)N * K * 2};
-  cuuint32_t box[3] = {64, ffn::BK, 1};
+  cuuint32_t box[3] = {64, BK, 1};
   cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -37,12 +36,12 @@ bool make_weight_map(CUtensorMap* map, const void* base, int E, int K, int N) {
 }
 
 // bf16 activations [rows, K] row-major: box = 64 (K) x 128 rows
-bool make_act_map(CUtensorMap* map, const void* base, int rows, int K) {
-  ffn::EncodeTiledFn fn = encode_fn();
+bool make_act_map(CUtensorMap* map, const void* base, long long rows, int K) {
+  EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-  cuuint32_t box[2] = {ffn::BK, ffn::BM};
+  cuuint32_t box[2] = {BK, BM};
   cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -51,7 +50,7 @@ bool make_act_map(CUtensorMap* map, const void* base, int rows, int K) {
 
 // E4M3 weights [E, N, K] (K contiguous): box = 128 bytes of K x 128 output columns x 1, 128-byte swizzle
 bool make_weight_map_fp8(CUtensorMap* map, const void* base, int E, int N, int K) {
-  ffn::EncodeTiledFn fn = encode_fn();
+  EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)N, (cuuint64_t)E};
   cuuint64_t strides[2] = {(cuuint64_t)K, (cuuint64_t)N * K};
@@ -64,18 +63,50 @@ bool make_weight_map_fp8(CUtensorMap* map, const void* base, int E, int N, int K
 
 // E4M3 activations [rows, K]: box = 128 bytes of K x 128 rows
 bool make_act_map_fp8(CUtensorMap* map, const void* base, int rows, int K) {
-  ffn::EncodeTiledFn fn = encode_fn();
+  EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
   cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)K};
-  cuuint32_t box[2] = {128, ffn::BM};
+  cuuint32_t box[2] = {128, BM};
   cuuint32_t estr[2] = {1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-}  // namespace
+// bf16 weights [E, K, N] read as the TRANSPOSED operand of a backward GEMM: the same memory seen as [E, N' = K, K' = N]
+// with K' contiguous; box = 64 (K') x 128 (N') x 1, 128-byte swizzle.  `rows` = N', `cols` = K'.
+bool make_weight_map_kmajor(CUtensorMap* map, const void* base, int E, int rows, int cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)E};
+  cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)rows * cols * 2};
+  cuuint32_t box[3] = {64, 128, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// bf16 rows [rows, cols] read with the row index as K (weight gradients): box = 64 columns x 64 rows
+bool make_rows_map_mn(CUtensorMap* map, const void* base, long long rows, int cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {64, 64};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace ffn
+
+using ffn::make_weight_map;
+using ffn::make_act_map;
+using ffn::make_weight_map_fp8;
+using ffn::make_act_map_fp8;
 
 int current_device() {
   int dev = 0;

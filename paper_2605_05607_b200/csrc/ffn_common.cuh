@@ -38,6 +38,11 @@ struct GemmParams {
   const float* b_scale2;        // [E, N]   (GEMM-1: W3)
   float* y_acc;                 // GEMM-2 with Combine in its epilogue: fp32 [T, N] accumulator, token
   int y_div;                    // of row r = row_pair[r] / y_div (NULL: rows go to `out`)
+  // backward pass (pair kernel modes PAIR_GLU_BWD / PAIR_KSPLIT)
+  const __nv_bfloat16* dh;      // [rows, N] incoming gradient of h (same leading dimension as out)
+  __nv_bfloat16* out2;          // dA1 [rows, N]
+  __nv_bfloat16* out3;          // dA3 [rows, N]
+  int k_split;                  // k-blocks taken from each of the two (A, B) pairs
 };
 
 struct Tile {
@@ -142,6 +147,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// tensor maps (ffn.cu)
+bool make_weight_map(CUtensorMap* map, const void* base, int E, int K, int N);
+bool make_act_map(CUtensorMap* map, const void* base, long long rows, int K);
+bool make_weight_map_fp8(CUtensorMap* map, const void* base, int E, int N, int K);
+bool make_act_map_fp8(CUtensorMap* map, const void* base, int rows, int K);
+bool make_weight_map_kmajor(CUtensorMap* map, const void* base, int E, int rows, int cols);
+bool make_rows_map_mn(CUtensorMap* map, const void* base, long long rows, int cols);
+cudaError_t launch_wgrad(const CUtensorMap& m_a, const CUtensorMap& m_b, const int32_t* poff, void* dw, int E, int M,
+                         int N, int32_t* status, cudaStream_t st);
+
 // fp8 = false: bf16 operands, weights [E, K, N] (B MN-major).  fp8 = true: E4M3 operands, weights
 // [E, N, K] (B K-major), 128 elements of K per pipeline stage, scales applied in the epilogue.
 cudaError_t launch_gemm1(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, bool fp8,
@@ -150,6 +165,11 @@ cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUt
                          cudaStream_t st);
 cudaError_t launch_gemm1_pair(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3,
                               const CUtensorMap& m_xs, cudaStream_t st);
+cudaError_t launch_bwd_dh(const GemmParams& p, const CUtensorMap& m_w2t, const CUtensorMap& m_do, cudaStream_t st);
+cudaError_t launch_bwd_glu(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, const CUtensorMap& m_xs,
+                           cudaStream_t st);
+cudaError_t launch_bwd_dx(const GemmParams& p, const CUtensorMap& m_w1t, const CUtensorMap& m_w3t, const CUtensorMap& m_da1,
+                          const CUtensorMap& m_da3, cudaStream_t st);
 size_t fused_max_blocks(int T, int k, int E);   // capacity of blk_start (+1) / blk_info for a shape
 size_t fused_tracker_words(int T, int k, int E);   // int32 words of the tracker region (dacc | done | tbcnt2 | nready | queue)
 cudaError_t launch_ffn_fused(FusedParams p, const int32_t* expert_counts, int32_t* blk_start, int4* blk_info,

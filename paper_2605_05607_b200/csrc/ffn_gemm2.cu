@@ -45,6 +45,7 @@ constexpr int SMEM_BYTES =
 constexpr int THREADS = 192;
 constexpr uint32_t IDESC = idesc_bf16(2 * BM);
 constexpr uint32_t IDESC_F8 = idesc_e4m3(2 * BM);
+constexpr uint32_t IDESC_BK = idesc_bf16(2 * BM) & ~(1u << 16);   // bf16 with a K-major B operand
 constexpr uint32_t HINT = 4000;   // try_wait suspend-time hint (ns), see ptx::mbar_try_wait
 
 // RED = false: rows go to o (bf16), Combine is a later pass.  RED = true: Combine happens here
@@ -53,13 +54,27 @@ constexpr uint32_t HINT = 4000;   // try_wait suspend-time hint (ns), see ptx::m
 // FP8 = true: h rows and weights are E4M3 codes, a stage holds 128 elements of K (the same 128 bytes
 // per row), W2 comes K-major from [E, N, K] as one 128-row box per CTA, and the epilogue applies
 // a_scale[row] * b_scale[e, n] together with the gate weight.
-// GLU = true: GEMM-1 with the SwiGLU epilogue (see the head of this file): map_b0 = W1, map_b1 = W3, 128 output
-// columns per tile; otherwise map_b0 = map_b1 = W2 and CTA `rank` takes columns n0 + 128 * rank.
-template <bool RED, bool FP8, bool GLU>
+// MODE selects the epilogue and the operand walk:
+//   PAIR_PLAIN    o = row weight x acc (GEMM-2; also dH = dO . W2^T of the backward pass): map_b0 = map_b1 = the weight,
+//                 CTA `rank` takes columns n0 + 128 * rank
+//   PAIR_GLU      GEMM-1 with the SwiGLU epilogue (see the head of this file): map_b0 = W1, map_b1 = W3, 128 output
+//                 columns per tile
+//   PAIR_GLU_BWD  the same GEMM recomputed in the backward pass: from a1 = a.W1, a3 = a.W3 and the incoming dh tile the
+//                 epilogue writes h, da1 = dh * a3 * silu'(a1) and da3 = dh * silu(a1)
+//   PAIR_KSPLIT   acc = A0 . B0 + A1 . B1 (dX = dA1 . W1^T + dA3 . W3^T): the first p.k_split k-blocks come from
+//                 (map_h, map_b0), the rest from (map_a1, map_b1); plain epilogue
+// BKMAJ: the bf16 weight operand is read K-major (one box of 128 columns x 64 K per CTA and stage), which is how
+// W^T looks when W is stored [K, N] with N contiguous: the backward GEMMs read the forward weights in place.
+enum { PAIR_PLAIN = 0, PAIR_GLU = 1, PAIR_GLU_BWD = 2, PAIR_KSPLIT = 3 };
+
+template <bool RED, bool FP8, int MODE, bool BKMAJ>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
-                 const __grid_constant__ CUtensorMap map_h, const GemmParams p) {
-  static_assert(!(GLU && (RED || FP8)), "the SwiGLU form exists for bf16 operands and row output only");
+                 const __grid_constant__ CUtensorMap map_h, const __grid_constant__ CUtensorMap map_a1,
+                 const GemmParams p) {
+  constexpr bool GLU = MODE == PAIR_GLU || MODE == PAIR_GLU_BWD;
+  constexpr bool KMAJ = FP8 || BKMAJ;   // the weight operand is K-major in shared memory
+  static_assert(!(MODE != PAIR_PLAIN && (RED || FP8)), "only the plain form has the reducing / FP8 variants");
   constexpr int BN_OUT = GLU ? 128 : 256;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -97,6 +112,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
     ptx::prefetch_tensormap(&map_b0);
     ptx::prefetch_tensormap(&map_b1);
     ptx::prefetch_tensormap(&map_h);
+    if (MODE == PAIR_KSPLIT) ptx::prefetch_tensormap(&map_a1);
   }
   if (warp == 5) {
     ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), 512);
@@ -115,7 +131,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
   const uint32_t tmem_base = *tmem_slot;
   const int total = tp_s[p.E] * p.n_tiles;
   constexpr int BK_ELEMS = FP8 ? 2 * BK : BK;   // K elements per stage: 128 bytes per row either way
-  const int KB = (p.K + BK_ELEMS - 1) / BK_ELEMS;
+  const int KB = MODE == PAIR_KSPLIT ? 2 * p.k_split : (p.K + BK_ELEMS - 1) / BK_ELEMS;
   volatile int* abort_flag = abort_s;
   const volatile int* global_abort = p.status + ST_ABORT;
 
@@ -140,7 +156,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UMMA_N);
       float* yrow = nullptr;
       float wr = 1.f;
-      if (valid && !GLU) {
+      if (valid && !GLU && (RED || p.topk_w != nullptr)) {
         const int pair = __ldg(p.row_pair + grow);
         if (p.topk_w != nullptr) wr = __ldg(p.topk_w + pair);
         if (FP8) wr *= __ldg(p.a_scale + grow);   // row scale of h joins the gate weight
@@ -158,7 +174,52 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
         }
         __syncwarp();
       }
-      if (GLU) {
+      if (MODE == PAIR_GLU_BWD) {
+        // backward of SwiGLU on the recomputed pre-activations: a thread owns one row and walks its 128 columns 32 at
+        // a time; dh comes from global memory (64 bytes of the row per step), h / da1 / da3 go straight back
+        const size_t rowoff = grow * (size_t)p.out_ld + t.n0;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t a1[32], a3[32];
+          ptx::tmem_ld32(taddr + c * 32, a1);
+          ptx::tmem_ld32(taddr + 128 + c * 32, a3);
+          ptx::tmem_ld_wait();
+          if (valid) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+              const int col = t.n0 + c * 32 + v * 8;
+              if (col < p.N) {
+                const size_t at = rowoff + c * 32 + v * 8;
+                const uint4 dq = *reinterpret_cast<const uint4*>(p.dh + at);
+                const __nv_bfloat162* dp = reinterpret_cast<const __nv_bfloat162*>(&dq);
+                uint32_t qh[4], q1[4], q3[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const int j = v * 8 + 2 * i;
+                  const float2 dhv = __bfloat1622float2(dp[i]);
+                  float hh[2], d1[2], d3[2];
+#pragma unroll
+                  for (int u = 0; u < 2; ++u) {
+                    const float x1 = __uint_as_float(a1[j + u]), x3 = __uint_as_float(a3[j + u]);
+                    const float dv = u ? dhv.y : dhv.x;
+                    const float sg = __fdividef(1.f, 1.f + __expf(-x1));
+                    const float sl = x1 * sg;
+                    hh[u] = sl * x3;
+                    d3[u] = dv * sl;
+                    d1[u] = dv * x3 * (sg * (1.f + x1 * (1.f - sg)));
+                  }
+                  qh[i] = pack2(hh[0], hh[1]);
+                  q1[i] = pack2(d1[0], d1[1]);
+                  q3[i] = pack2(d3[0], d3[1]);
+                }
+                *reinterpret_cast<uint4*>(p.out + at) = make_uint4(qh[0], qh[1], qh[2], qh[3]);
+                *reinterpret_cast<uint4*>(p.out2 + at) = make_uint4(q1[0], q1[1], q1[2], q1[3]);
+                *reinterpret_cast<uint4*>(p.out3 + at) = make_uint4(q3[0], q3[1], q3[2], q3[3]);
+              }
+            }
+          }
+        }
+      } else if (GLU) {
         // SwiGLU of the W1 half (columns 0..127) and the W3 half (128..255): 128 columns of h, transposed
         // through shared memory 64 columns at a time and stored as whole 128-byte row segments
         const uint32_t stage = stage_base + (uint32_t)(warp * STAGE_OUT_WARP);
@@ -296,11 +357,12 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
           const uint32_t lead_full = ptx::mapa(full_bar(s), 0);
           // the leader announces the bytes of both CTAs; the peer's copies only complete them
           if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
-          const int k0 = kb * BK_ELEMS;
-          ptx::tma_load_2d_pair(sa, &map_h, lead_full, k0, t.row0);
-          const CUtensorMap* map_b = rank == 0 ? &map_b0 : &map_b1;
+          const bool second = MODE == PAIR_KSPLIT && kb >= p.k_split;     // second (A, B) pair of the K walk
+          const int k0 = (second ? kb - p.k_split : kb) * BK_ELEMS;
+          ptx::tma_load_2d_pair(sa, second ? &map_a1 : &map_h, lead_full, k0, t.row0);
+          const CUtensorMap* map_b = MODE == PAIR_KSPLIT ? (second ? &map_b1 : &map_b0) : (rank == 0 ? &map_b0 : &map_b1);
           const int nb = GLU ? t.n0 : t.n0 + rank * 128;   // this CTA's 128 columns of the B tile
-          if (FP8) {   // one K-major box: this CTA's 128 output columns x 128 bytes of K
+          if (KMAJ) {   // one K-major box: this CTA's 128 output columns x 128 bytes of K
             ptx::tma_load_3d_pair(sb, map_b, lead_full, k0, nb, t.e);
           } else {     // two MN-major slabs of 64 output columns x 64 rows of K
             ptx::tma_load_3d_pair(sb, map_b, lead_full, nb, k0, t.e);
@@ -314,7 +376,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
     // ================================ UMMA issuer (leader CTA only) ================================
     if (rank == 0 && lane == 0) {
       const uint64_t a_base = desc_base(16, 1024);
-      const uint64_t b_base = FP8 ? desc_base(16, 1024) : desc_base(BK * 128, 1024);   // K-major : MN-major
+      const uint64_t b_base = KMAJ ? desc_base(16, 1024) : desc_base(BK * 128, 1024);   // K-major : MN-major
       uint32_t it = 0;
       int tl = 0;
       for (int w = cluster_id; w < total && !*abort_flag; w += num_clusters, ++tl) {
@@ -336,6 +398,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
 #pragma unroll
           for (int k = 0; k < 4; ++k) {   // 32 bytes of K per UMMA (16 bf16 / 32 E4M3): +32 B inside the swizzle row
             if (FP8) ptx::umma_f8_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), IDESC_F8, (kb | k) != 0);
+            else if (BKMAJ) ptx::umma_bf16_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), IDESC_BK, (kb | k) != 0);
             else ptx::umma_bf16_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), IDESC, (kb | k) != 0);   // B: +2 atoms
           }
           // free the stage in both CTAs once these UMMAs have read it
@@ -380,7 +443,7 @@ int pair_grid() {
     attr.val.clusterDim.z = 1;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    if (cudaOccupancyMaxActiveClusters(&clusters, ffn_gemm2_kernel<false, false, false>, &cfg) != cudaSuccess || clusters <= 0) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, ffn_gemm2_kernel<false, false, PAIR_PLAIN, false>, &cfg) != cudaSuccess || clusters <= 0) {
       (void)cudaGetLastError();
       clusters = sm_count() / 2;
     }
@@ -399,11 +462,14 @@ cudaError_t set_pair_attributes() {
   const int dev = current_device();
   if (!attr_set[dev].load(std::memory_order_acquire)) {
     const auto attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
-    cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, false>, attr, SMEM_BYTES);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, false, false>, attr, SMEM_BYTES);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, true, false>, attr, SMEM_BYTES);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, true, false>, attr, SMEM_BYTES);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, true>, attr, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, PAIR_PLAIN, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, false, PAIR_PLAIN, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, true, PAIR_PLAIN, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<true, true, PAIR_PLAIN, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, PAIR_GLU, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, PAIR_PLAIN, true>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, PAIR_GLU_BWD, false>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, PAIR_KSPLIT, true>, attr, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set[dev].store(true, std::memory_order_release);
   }
@@ -417,12 +483,13 @@ cudaError_t launch_gemm2(const GemmParams& p, const CUtensorMap& m_w2, const CUt
   if (e != cudaSuccess) return e;
   ProfileScope prof(KID_GEMM2, st);
   const bool red = p.y_acc != nullptr;
+  const int g = pair_grid();
   if (fp8) {
-    if (red) return launch_pdl(ffn_gemm2_kernel<true, true, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, p);
-    return launch_pdl(ffn_gemm2_kernel<false, true, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, p);
+    if (red) return launch_pdl(ffn_gemm2_kernel<true, true, PAIR_PLAIN, false>, g, THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, m_h, p);
+    return launch_pdl(ffn_gemm2_kernel<false, true, PAIR_PLAIN, false>, g, THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, m_h, p);
   }
-  if (red) return launch_pdl(ffn_gemm2_kernel<true, false, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, p);
-  return launch_pdl(ffn_gemm2_kernel<false, false, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, p);
+  if (red) return launch_pdl(ffn_gemm2_kernel<true, false, PAIR_PLAIN, false>, g, THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, m_h, p);
+  return launch_pdl(ffn_gemm2_kernel<false, false, PAIR_PLAIN, false>, g, THREADS, SMEM_BYTES, st, m_w2, m_w2, m_h, m_h, p);
 }
 
 // GEMM-1 on CTA pairs: m_xs maps the expert-sorted activation rows [P, K]; p.tile_prefix = the 256-row pair-tile
@@ -432,7 +499,33 @@ cudaError_t launch_gemm1_pair(const GemmParams& p, const CUtensorMap& m_w1, cons
   cudaError_t e = set_pair_attributes();
   if (e != cudaSuccess) return e;
   ProfileScope prof(KID_GEMM1, st);
-  return launch_pdl(ffn_gemm2_kernel<false, false, true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w1, m_w3, m_xs, p);
+  return launch_pdl(ffn_gemm2_kernel<false, false, PAIR_GLU, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w1, m_w3, m_xs,
+                    m_xs, p);
+}
+
+// Backward pass, all on CTA pairs (see bwd.cu for the sequence):
+//   launch_bwd_dh    dh = dO . W2^T          A = dO rows (m_do), B = W2 read K-major (m_w2t), N = f, K = d
+//   launch_bwd_glu   GEMM-1 recomputed with the backward SwiGLU epilogue: p.dh in, p.out = h, p.out2 = dA1, p.out3 = dA3
+//   launch_bwd_dx    dXs = dA1 . W1^T + dA3 . W3^T   A = (m_da1, m_da3), B = (m_w1t, m_w3t) K-major, p.k_split k-blocks each
+cudaError_t launch_bwd_dh(const GemmParams& p, const CUtensorMap& m_w2t, const CUtensorMap& m_do, cudaStream_t st) {
+  cudaError_t e = set_pair_attributes();
+  if (e != cudaSuccess) return e;
+  return launch_pdl(ffn_gemm2_kernel<false, false, PAIR_PLAIN, true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w2t, m_w2t,
+                    m_do, m_do, p);
+}
+cudaError_t launch_bwd_glu(const GemmParams& p, const CUtensorMap& m_w1, const CUtensorMap& m_w3, const CUtensorMap& m_xs,
+                           cudaStream_t st) {
+  cudaError_t e = set_pair_attributes();
+  if (e != cudaSuccess) return e;
+  return launch_pdl(ffn_gemm2_kernel<false, false, PAIR_GLU_BWD, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_w1, m_w3,
+                    m_xs, m_xs, p);
+}
+cudaError_t launch_bwd_dx(const GemmParams& p, const CUtensorMap& m_w1t, const CUtensorMap& m_w3t, const CUtensorMap& m_da1,
+                          const CUtensorMap& m_da3, cudaStream_t st) {
+  cudaError_t e = set_pair_attributes();
+  if (e != cudaSuccess) return e;
+  return launch_pdl(ffn_gemm2_kernel<false, false, PAIR_KSPLIT, true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w1t, m_w3t,
+                    m_da1, m_da3, p);
 }
 
 }  // namespace ffn

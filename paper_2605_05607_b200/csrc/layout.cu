@@ -323,6 +323,12 @@ static int row_parts(int T, int vec_per_row) {
 
 cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
                            const float* topk_w, void* pg, void* y, int32_t* status, cudaStream_t st) {
+  return launch_combine_rows(s, o, L, topk_idx, topk_w, pg, y, s.T * s.k, status, st);
+}
+
+// n_rows: rows of `o` (L.pair_row entries outside [0, n_rows) are reported and skipped)
+cudaError_t launch_combine_rows(const Shape& s, const void* o, const Layout& L, const int32_t* topk_idx,
+                                const float* topk_w, void* pg, void* y, int n_rows, int32_t* status, cudaStream_t st) {
   if (s.T == 0) return cudaSuccess;
   const int vec = s.d / 8;
   const int parts = row_parts(s.T, vec);
@@ -333,7 +339,7 @@ cudaError_t launch_combine(const Shape& s, const void* o, const Layout& L, const
   ProfileScope prof(KID_COMBINE, st);
   CombineArgs c{static_cast<const uint4*>(o), static_cast<uint4*>(y), static_cast<uint4*>(pg), topk_idx, topk_w,
                 L.pair_row, L.al, L.group_offsets, s.T, s.E, s.k, s.E / s.G, vec, (s.flags & 1) ? 1 : 0,
-                s.T * s.k, status};
+                n_rows, status};
   if (s.k <= 2) return launch_pdl(combine_kernel<2>, (unsigned)blocks, 256, 0, st, c, parts, vec_per_part);
   if (s.k <= 4) return launch_pdl(combine_kernel<4>, (unsigned)blocks, 256, 0, st, c, parts, vec_per_part);
   return launch_pdl(combine_kernel<8>, (unsigned)blocks, 256, 0, st, c, parts, vec_per_part);
