@@ -278,12 +278,14 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
     def layer_single_kernel_ffn():
         B.moe_layer(shape_trk, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws)
 
+    # the variants alternate and the order flips every repetition: at the power cap a call inherits the clock state
+    # its predecessor left, so a fixed order would favour whoever runs after the cheapest call
     seq_ms, fus_ms, epi_ms, trk_ms = [], [], [], []
-    for _ in range(reps):
-        seq_ms.append(timed(unfused_seq))
-        fus_ms.append(timed(calls["layer_fused"]))
-        epi_ms.append(timed(layer_epilogue_combine))
-        trk_ms.append(timed(layer_single_kernel_ffn))
+    order = [(seq_ms, unfused_seq), (fus_ms, calls["layer_fused"]), (epi_ms, layer_epilogue_combine),
+             (trk_ms, layer_single_kernel_ffn)]
+    for rep in range(2 * reps):
+        for acc, fn in (order if rep % 2 == 0 else order[::-1]):
+            acc.append(timed(fn))
     # in-layer (back to back, no idle gap) kernel times of the fused call
     for kn in kernels["layer_fused"]:
         B.moe_profile_enable(B.KERNEL_IDS[kn])
@@ -336,6 +338,52 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
                       "rows_per_expert_min": int(counts.min()), "rows_per_expert_max": int(counts.max()),
                       "empty_experts": int((counts == 0).sum()), "timing": "cold L2 (512 MB overwritten, then 256 MB of it read back, before each call)"}
     return out
+
+
+def backward_leg(cfg, t, reps=5):
+    """moe_layer_backward (fixed routing from the forward) on the same workload: device time per call, and the
+    training step (forward + backward) it gives.  Useful flops: 12 P d f of gradient GEMMs + 4 P d f of GEMM-1
+    recomputed for its pre-activations."""
+    from paper_2605_05607_b200 import binding as B
+    shape = B.make_shape(cfg)
+    ws = B.alloc_workspace(shape)
+    T, E, d, f, P = cfg.T, cfg.E, cfg.d, cfg.f, cfg.P
+    dev = "cuda"
+    idx = torch.zeros(P, dtype=torch.int32, device=dev)
+    w = torch.zeros(P, dtype=torch.float32, device=dev)
+    lay = B.alloc_layout(shape)
+    y = torch.zeros(T, d, dtype=torch.bfloat16, device=dev)
+    dy = torch.randn(T, d, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    dx = torch.empty_like(y)
+    dw1, dw3, dw2 = torch.empty_like(t["w1"]), torch.empty_like(t["w3"]), torch.empty_like(t["w2"])
+    bws = torch.zeros(B.moe_backward_workspace_bytes(shape), dtype=torch.uint8, device=dev)
+
+    def fwd():
+        B.moe_layer(shape, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws, topk_idx=idx, topk_w=w,
+                    layout=lay)
+
+    def bwd():
+        B.moe_layer_backward(shape, t["x"], dy, idx, w, lay, t["w1"], t["w3"], t["w2"], dx, dw1, dw3, dw2, bws)
+
+    def timed(fn, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    fwd(); bwd()
+    torch.cuda.synchronize()
+    assert B.moe_status(bws)[0] == 0
+    f_ms, b_ms = timed(fwd, reps), timed(bwd, reps)
+    step_ms = timed(lambda: (fwd(), bwd()), reps)
+    assert B.moe_status(bws)[0] == 0 and B.moe_status(ws)[0] == 0
+    return {"backward_ms": b_ms, "forward_ms": f_ms, "training_step_ms": step_ms,
+            "training_tokens_per_s": T / step_ms * 1e3, "backward_tflops": 16.0 * P * d * f / b_ms / 1e9,
+            "flops_counted": "12 P d f gradient GEMMs + 4 P d f recomputed GEMM-1", "reps": reps,
+            "routing": "fixed (expert indices and gate weights of the forward; the gate's own gradient is outside)"}
 
 
 def workload_config(cfg, n_gpus):
@@ -424,6 +472,7 @@ def main():
                          "gloo backend (no GPU, no library); prints the JSON line's n_gpus / steps / ms_per_step")
     ap.add_argument("--lean", action="store_true",
                     help="timed region only: no e2e / stage / cpu_baseline legs (for profiler captures)")
+    ap.add_argument("--no-backward", action="store_true", help="skip the backward / training-step leg")
     ap.add_argument("--stages-only", action="store_true",
                     help="only the per-stage breakdown of --config (prints its JSON); for profiler captures")
     ap.add_argument("--no-ffn", action="store_true", help="with --stages-only: skip expert weights and the FFN")
@@ -621,6 +670,14 @@ def main():
             clocks["window"] = "same load repeated for 1.5 s after the timed region"
         sampler.stop()
 
+    ep_wire = None
+    if ep_rank is not None:     # rows and bytes every rank sends per layer, with and without the per-group de-duplication
+        mine = ep_rank.wire_stats()
+        ep_wire = [mine]
+        if world > 1:
+            ep_wire = [None] * world
+            dist.all_gather_object(ep_wire, mine)
+
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -681,6 +738,7 @@ def main():
     if args.layer_flags:
         line["config"]["layer_flags"] = args.layer_flags
     if ep_rank is not None:
+        line["ep_wire_per_rank"] = ep_wire
         line["config"]["parallelism"] = (f"expert parallel x{world}: {cfg.m} experts per GPU, all-to-all of one row per "
                                          "(token, group) out and one pre-reduced row back; split sizes read back once per layer")
         line["stages"] = None
@@ -703,6 +761,8 @@ def main():
                                                                           "frac_bf16_burst", "frac_bf16_sustained")}
         line["fused_vs_unfused_ms"] = {k: st["summary"][k] for k in ("fused_back_to_back_ms", "unfused_back_to_back_ms",
                                                                       "fused_ms", "unfused_sum_ms")}
+    if world == 1 and not args.lean and ep_rank is None and not fp8 and not args.no_backward:
+        line["backward"] = backward_leg(cfg, t)
     if world == 1 and args.report and not args.lean:
         report = {cfg.name: line["stages"]}
         del t

@@ -89,7 +89,12 @@ enum { MOE_FLAG_WEIGHT_IN_COMBINE = 1,   /* default (0): gate weight applied in 
                                             layout tensors of Sec. III-D (one dense row per (token, expert), expert-
                                             sorted, in the workspace) and GEMM-1 reads them as TMA tiles on CTA pairs
                                             (cta_group::2, 256-row tiles) instead of gathering token rows inside
-                                            the GEMM.  Same h as the gathering form.  Excludes MOE_FLAG_FUSED_FFN.     */
+                                            the GEMM.  Same h as the gathering form, bit for bit.  Without this flag
+                                            and without MOE_FLAG_GEMM1_GATHER the library takes this form by itself
+                                            for wide experts (f >= 8192, at least 512 rows per expert on average),
+                                            where the extra pass over the rows costs less than it gains.  Excludes
+                                            MOE_FLAG_FUSED_FFN and MOE_FLAG_GEMM1_GATHER.                              */
+       MOE_FLAG_GEMM1_GATHER = 512,      /* GEMM-1 always gathers token rows itself (cta_group::1, 128-row tiles)   */
        MOE_FLAG_TRACK_DISPATCH = 256,    /* with MOE_FLAG_FUSED_FFN: Dispatch runs as tasks of the same kernel.  Worker
                                             warps write the per-expert layout tensors (Sec. III-D) 16 rows at a time and
                                             count them in the Tile Status table (DAcc, Sec. IV-B); a GEMM-1 tile starts

@@ -39,6 +39,7 @@ MOE_FLAG_GEMM2_PAIR = 32
 MOE_FLAG_GEMM2_SINGLE = 64
 MOE_FLAG_GEMM1_PAIR = 128
 MOE_FLAG_TRACK_DISPATCH = 256
+MOE_FLAG_GEMM1_GATHER = 512
 
 EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "moe_status", "moe_strerror",
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",

@@ -24,6 +24,17 @@ struct WsPlan {
   int W;
 };
 
+// GEMM-1 form.  The CTA-pair form needs the per-expert layout tensors (one more pass over P rows of d) and runs
+// GEMM-1 about 8 % faster; the pass costs about 240 / f of GEMM-1's time, so it pays for wide experts.  Taken when asked
+// for (MOE_FLAG_GEMM1_PAIR), or by itself for f >= 8192 with experts of at least 512 rows on average (measured: the
+// Mixtral-shaped layer gains 3 %, f = 1536 and f = 2048 layers lose 1-6 %); MOE_FLAG_GEMM1_GATHER keeps the gathering
+// form.  bf16 experts outside the tracker-paced kernel only.
+bool pair_gemm1(const moe_shape_t& s) {
+  if (s.flags & (MOE_FLAG_FUSED_FFN | MOE_FLAG_GEMM1_GATHER)) return false;
+  if (s.flags & MOE_FLAG_GEMM1_PAIR) return true;
+  return s.f >= 8192 && (long long)s.T * s.k >= 512ll * s.E;
+}
+
 WsPlan plan(const moe_shape_t& s) {
   WsPlan p{};
   const size_t T = (size_t)s.T, E = (size_t)s.E, G = (size_t)s.G, k = (size_t)s.k;
@@ -55,7 +66,7 @@ WsPlan plan(const moe_shape_t& s) {
   }
   p.wsplit = take(gate_split_bytes(s.d, s.E));
   // expert-sorted activation rows of the CTA-pair GEMM-1 (only reserved when that form is asked for)
-  p.xs = take((s.flags & (MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH)) ? P * (size_t)s.d * 2 : 0);
+  p.xs = take((pair_gemm1(s) || (s.flags & MOE_FLAG_TRACK_DISPATCH)) ? P * (size_t)s.d * 2 : 0);
   p.h = take(P * (size_t)s.f * 2);
   p.hq = take(P * (size_t)s.f);   // FP8 form: E4M3 copy of h and its row scales
   p.sh = take(P * 4);
@@ -84,10 +95,11 @@ int check_shape(const moe_shape_t* s) {
   if (s->T < 0 || s->d <= 0 || s->f <= 0 || s->E <= 0 || s->k <= 0 || s->G <= 0) return MOE_ERR_INVALID_ARG;
   if (s->score_fn != MOE_SCORE_SOFTMAX && s->score_fn != MOE_SCORE_SIGMOID) return MOE_ERR_INVALID_ARG;
   if (s->flags & ~(MOE_FLAG_WEIGHT_IN_COMBINE | MOE_FLAG_COMBINE_IN_EPILOGUE | MOE_FLAG_SPARSE_TOPK | MOE_FLAG_FUSED_FFN |
-                   MOE_FLAG_SM_PARTITION | MOE_FLAG_GEMM2_PAIR | MOE_FLAG_GEMM2_SINGLE | MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH))
+                   MOE_FLAG_SM_PARTITION | MOE_FLAG_GEMM2_PAIR | MOE_FLAG_GEMM2_SINGLE | MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH |
+                   MOE_FLAG_GEMM1_GATHER))
     return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_GEMM2_PAIR) && (s->flags & MOE_FLAG_GEMM2_SINGLE)) return MOE_ERR_INVALID_ARG;
-  if ((s->flags & MOE_FLAG_GEMM1_PAIR) && (s->flags & MOE_FLAG_FUSED_FFN)) return MOE_ERR_INVALID_ARG;
+  if ((s->flags & MOE_FLAG_GEMM1_PAIR) && (s->flags & (MOE_FLAG_FUSED_FFN | MOE_FLAG_GEMM1_GATHER))) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_SM_PARTITION) && !(s->flags & MOE_FLAG_FUSED_FFN)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_TRACK_DISPATCH) && !(s->flags & MOE_FLAG_FUSED_FFN)) return MOE_ERR_INVALID_ARG;
   if ((s->flags & MOE_FLAG_FUSED_FFN) && (s->flags & MOE_FLAG_COMBINE_IN_EPILOGUE)) return MOE_ERR_INVALID_ARG;
@@ -429,7 +441,8 @@ int moe_expert_ffn(const moe_shape_t* shape, const void* xg, const moe_layout_t*
   a.w1 = w1;
   a.w3 = w3;
   a.w2 = w2;
-  a.xs = (shape->flags & (MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH)) ? at<void>(ws, p.xs) : nullptr;
+  a.xs = (pair_gemm1(*shape) || (shape->flags & MOE_FLAG_TRACK_DISPATCH)) ? at<void>(ws, p.xs) : nullptr;
+  a.pair_gemm1 = pair_gemm1(*shape);
   a.track_dispatch = (shape->flags & MOE_FLAG_TRACK_DISPATCH) != 0;
   a.h = at<void>(ws, p.h);
   a.o = o;
@@ -586,7 +599,8 @@ int moe_expert_ffn_fp8(const moe_shape_t* shape, const void* xq, const float* sx
   a.w1 = w1q;
   a.w3 = w3q;
   a.w2 = w2q;
-  a.xs = (shape->flags & (MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH)) ? at<void>(ws, p.xs) : nullptr;
+  a.xs = (pair_gemm1(*shape) || (shape->flags & MOE_FLAG_TRACK_DISPATCH)) ? at<void>(ws, p.xs) : nullptr;
+  a.pair_gemm1 = pair_gemm1(*shape);
   a.track_dispatch = (shape->flags & MOE_FLAG_TRACK_DISPATCH) != 0;
   a.h = at<void>(ws, p.h);
   a.o = o;
@@ -693,7 +707,8 @@ static int layer_impl(const moe_shape_t* shape, const void* x, const float* w_ga
   a.w1 = w1;
   a.w3 = w3;
   a.w2 = w2;
-  a.xs = (shape->flags & (MOE_FLAG_GEMM1_PAIR | MOE_FLAG_TRACK_DISPATCH)) ? at<void>(ws, p.xs) : nullptr;
+  a.xs = (pair_gemm1(*shape) || (shape->flags & MOE_FLAG_TRACK_DISPATCH)) ? at<void>(ws, p.xs) : nullptr;
+  a.pair_gemm1 = pair_gemm1(*shape);
   a.track_dispatch = (shape->flags & MOE_FLAG_TRACK_DISPATCH) != 0;
   a.h = at<void>(ws, p.h);
   a.o = at<void>(ws, p.o);

@@ -129,6 +129,7 @@ struct FfnArgs {
   int gather_div;
   const void *w1, *w3, *w2;
   void* xs;                   // [P, d] bf16 scratch: expert-sorted activation rows (CTA-pair GEMM-1), or NULL
+  bool pair_gemm1;            // GEMM-1 on CTA pairs from xs (the caller's flag or the shape rule)
   void* h;                    // [P, f] bf16 scratch
   void* o;                    // [P, d] bf16 out (unused when y_acc is set)
   float* y_acc;               // Combine in GEMM-2's epilogue: zeroed fp32 [T, d] accumulator, else NULL

@@ -207,8 +207,8 @@ cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st)
   g1.n_tiles = (s.f + 127) / 128;
   g1.status = a.status;
   cudaError_t err;
-  if ((s.flags & 128) && a.xs != nullptr) {
-    // flag bit 128 (MOE_FLAG_GEMM1_PAIR): Dispatch writes the per-expert layout tensors, GEMM-1 runs on CTA pairs
+  if (a.pair_gemm1 && a.xs != nullptr) {
+    // Dispatch writes the per-expert layout tensors, GEMM-1 runs on CTA pairs (MOE_FLAG_GEMM1_PAIR, or the shape rule)
     CUtensorMap m_xs;
     if (!make_act_map(&m_xs, a.xs, P, s.d)) return cudaErrorInvalidValue;
     if ((err = launch_permute_rows(s, a.a_src, a.a_rows, a.gather_idx, a.gather_div, a.expert_offsets, a.xs, a.status,

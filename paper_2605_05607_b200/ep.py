@@ -105,6 +105,12 @@ class EpRank:
         B.moe_ep_finish(self.shape, back, self.lay, self.y)
         return self.y[: self.cfg.T]
 
+    def wire_stats(self) -> Dict[str, float]:
+        """Link traffic of the last forward() / send_phase() of this rank (reads two small device arrays)."""
+        gc = self.lay.group_counts[: self.cfg.G].tolist()
+        ec = self.lay.expert_counts[: self.cfg.E].tolist()
+        return wire_stats(self.cfg, self.rank, gc, ec)
+
     def status(self) -> List[int]:
         return [B.moe_status(self.ws)[0]] + [B.moe_status(b["ws"])[0] for b in self._recv.values()]
 
@@ -119,6 +125,32 @@ class EpRank:
         partial = self.recv_phase(rows, idx, w)
         back = all_to_all_rows(partial, recv_counts, out.counts, group)
         return self.finish_phase(back)
+
+
+def wire_stats(cfg: MoEConfig, rank: int, group_counts: Sequence[int], expert_counts: Sequence[int]) -> Dict[str, float]:
+    """What one rank puts on the links for one layer, from the device counters of its dispatch layout (group g lives
+    on rank g; rows for the rank's own group never leave it).
+
+    * with the per-group de-duplication / pre-reduction (Sec. III-D: one copy per destination out, one reduced row per
+      destination back): `group_counts[g]` rows of d bf16 each way, plus the trimmed target list (kk local expert ids
+      and gate weights per row) on the way out;
+    * point to point (one copy per (token, expert) pair each way, what Sec. II-B calls redundant): the pairs whose
+      expert lives in group g, i.e. the sum of `expert_counts` over that group, plus one id and weight per row.
+
+    Returns rows and bytes for both and the share of bytes the de-duplication removes."""
+    m, d = cfg.m, cfg.d
+    kk = min(cfg.k, m)
+    rows_dedup = sum(int(c) for g, c in enumerate(group_counts) if g != rank)
+    rows_p2p = sum(int(sum(expert_counts[g * m:(g + 1) * m])) for g in range(cfg.G) if g != rank)
+    row_bytes = 2 * d
+    out_dedup = rows_dedup * (row_bytes + 8 * kk)
+    out_p2p = rows_p2p * (row_bytes + 8)
+    back_dedup, back_p2p = rows_dedup * row_bytes, rows_p2p * row_bytes
+    total_dedup, total_p2p = out_dedup + back_dedup, out_p2p + back_p2p
+    return {"rows_dedup": rows_dedup, "rows_point_to_point": rows_p2p,
+            "bytes_out_dedup": out_dedup, "bytes_back_dedup": back_dedup,
+            "bytes_out_point_to_point": out_p2p, "bytes_back_point_to_point": back_p2p,
+            "bytes_removed_share": 0.0 if total_p2p == 0 else 1.0 - total_dedup / total_p2p}
 
 
 def exchange_counts(send_counts: Sequence[int], group=None) -> List[int]:

@@ -79,8 +79,15 @@ def test_bad_flags_rejected(lib):
     with pytest.raises(B.MoEError) as ei:
         B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=3))
     assert ei.value.code == B.MOE_ERR_INVALID_ARG
-    for ok in (0, 1, 2, 4, 5, 8, 9, 24, 32, 64):
+    for bad in (128 | 8, 128 | 512, 256, 16):            # pair GEMM-1 inside the tracker kernel / with its opposite; options without their base flag
+        with pytest.raises(B.MoEError):
+            B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=bad))
+    for ok in (0, 1, 2, 4, 5, 8, 9, 24, 32, 64, 128, 512, 8 | 256, 8 | 16 | 256):
         assert B.moe_workspace_bytes(B.make_shape(synth.CONFIGS["C1"], flags=ok)) > 0
+    # the Mixtral-shaped layer takes the CTA-pair GEMM-1 by itself: its workspace holds the per-expert layout tensors
+    c2 = synth.CONFIGS["C2"]
+    assert (B.moe_workspace_bytes(B.make_shape(c2)) - B.moe_workspace_bytes(B.make_shape(c2, B.MOE_FLAG_GEMM1_GATHER))
+            >= c2.P * c2.d * 2)
     # k = 1: the fp32 token accumulators are larger than o and the workspace accounts for them
     c = synth.CONFIGS["C1"].with_(k=1)
     assert B.moe_workspace_bytes(B.make_shape(c)) >= c.T * c.d * 4 + c.T * c.f * 2

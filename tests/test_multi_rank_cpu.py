@@ -124,3 +124,47 @@ def test_bench_starts_its_own_ranks_and_reports_the_real_world_size():
                           "--steps", "1"], env=dict(env, WORLD_SIZE="1", RANK="0"), capture_output=True, text=True,
                          timeout=300)
     assert bad.returncode != 0 and "must agree" in bad.stderr
+
+
+def _ep_wire_worker(rank, world, port, out):
+    """Each rank routes its own tokens (uneven, skewed routing), builds the dispatch layout with the CPU oracle and
+    derives its link traffic from the layout's counters; the totals are summed over the ranks."""
+    import numpy as np
+    from oracle import moe_oracle as O
+    from paper_2605_05607_b200 import ep
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        cfg = synth.MoEConfig("epw", T=40 + 25 * rank, d=64, f=32, E=8, k=3, G=world, bias="zipf", zipf_s=1.3, seed=31 + rank)
+        rng = np.random.default_rng(100 + rank)
+        logits = rng.standard_normal((cfg.T, cfg.E)).astype(np.float32)
+        idx, _ = O.route(logits, synth.make_bias(cfg).numpy(), cfg.k, cfg.score_fn)
+        lay = O.layout(idx, cfg.E, cfg.G)
+        st = ep.wire_stats(cfg, rank, lay["group_counts"], lay["expert_counts"])
+        # brute force over every (token, slot): rows that leave this rank with and without the de-duplication
+        dests = [{int(e) // cfg.m for e in row} - {rank} for row in idx]
+        assert st["rows_dedup"] == sum(len(dd) for dd in dests)
+        assert st["rows_point_to_point"] == sum(1 for row in idx for e in row if int(e) // cfg.m != rank)
+        assert st["bytes_back_dedup"] == st["rows_dedup"] * 2 * cfg.d
+        assert 0.0 <= st["bytes_removed_share"] < 1.0 and st["rows_dedup"] <= st["rows_point_to_point"]
+        tot = torch.tensor([st["rows_dedup"], st["rows_point_to_point"]], dtype=torch.int64)
+        dist.all_reduce(tot)
+        dist.barrier()
+        if rank == 0:
+            out.put(tot.tolist())
+    finally:
+        dist.destroy_process_group()
+
+
+def test_ep_wire_bytes_with_and_without_dedup_on_uneven_routing():
+    world, port = 2, _free_port()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    procs = [ctx.Process(target=_ep_wire_worker, args=(r, world, port, q)) for r in range(world)]
+    for p in procs:
+        p.start()
+    dedup, p2p = q.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert 0 < dedup < p2p          # skewed top-3 over 2 groups of 4 experts: several experts of a token share a group
