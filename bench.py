@@ -34,7 +34,7 @@ KERNELS_PER_STEP = 10  # gate split, gate, topk, masks, scan, offsets, fill, gem
 
 NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16 data-sheet figure, for context beside the measured peaks
 BURST_REGION_S = 1.0           # a timed region shorter than this runs before the power cap settles: burst peak
-CPU_SAMPLE_TOKENS = 16         # tokens per oracle pass, the same for the cpu_baseline leg and the reference arm
+CPU_SAMPLE_TOKENS = 12         # tokens per oracle pass, the same for the cpu_baseline leg and the reference arm
 
 # DRAM bytes (read + write) of one GEMM-1 launch, dram__bytes_read.sum + dram__bytes_write.sum of a
 # single-pass ncu capture of that workload; absent: null in the line.

@@ -213,3 +213,23 @@ def test_fullsize_tracker_paced_layer_equals_the_separate_kernels(name):
             assert other.status()[0] == 0, (flags, other.status())
             assert torch.equal(other.y[: cfg.T], y_ref[: cfg.T]), flags
         del other
+
+
+def test_gemm1_is_bit_reproducible_over_many_runs():
+    """GEMM-1's gathered rows reach the tensor core through cp.async copies that arrive on the stage barrier by
+    themselves, with no proxy fence between the copies and the UMMA that reads them.  If that publication were not
+    sound, a row would now and then be multiplied before it had landed: twenty runs of the expert FFN on C4 (131 072
+    rows, 4 096-deep K) must give the same o bit for bit, and the first run is held to the oracle by the tests above."""
+    cfg = synth.ALL_CONFIGS["C4"]
+    run = H.Run(cfg, B.MOE_FLAG_GEMM1_GATHER)
+    run.route()
+    run.dispatch()
+    run.ffn()
+    torch.cuda.synchronize()
+    first = run.o.clone()
+    for i in range(20):
+        run.o.fill_(1.0)
+        run.ffn()
+        torch.cuda.synchronize()
+        assert torch.equal(run.o[: cfg.P], first[: cfg.P]), i
+    assert run.status()[0] == 0
