@@ -32,6 +32,20 @@ METRIC = "fused MoE layer tokens/sec"
 UNIT = "tokens/s"
 KERNELS_PER_STEP = 10  # gate split, gate, topk, masks, scan, offsets, fill, gemm1, gemm2, combine
 
+
+def kernels_per_step(cfg, flags: int, fp8: bool) -> int:
+    """Launches of one moe_layer call, following the library's own choice of forms (see MOE_FLAG_* in tcmoe.h)."""
+    from paper_2605_05607_b200 import binding as B
+    if flags & B.MOE_FLAG_FUSED_FFN:
+        return 7 + 2                                   # ... layout, then the task-table kernel and the tracker-paced kernel
+    n = KERNELS_PER_STEP + (2 if fp8 else 0)           # FP8: + quantisation of x and of h
+    if flags & B.MOE_FLAG_COMBINE_IN_EPILOGUE:
+        return n                                       # no combine kernel, one rounding pass instead
+    wide = cfg.f >= 8192 and cfg.T * cfg.k >= 512 * cfg.E
+    if not fp8 and not flags & B.MOE_FLAG_GEMM1_GATHER and (flags & B.MOE_FLAG_GEMM1_PAIR or wide):
+        n += 1                                         # the layout-tensor pass in front of the CTA-pair GEMM-1
+    return n
+
 NOMINAL_BF16_TFLOPS = 2250.0   # dense bf16 data-sheet figure, for context beside the measured peaks
 BURST_REGION_S = 1.0           # a timed region shorter than this runs before the power cap settles: burst peak
 CPU_SAMPLE_TOKENS = 12         # tokens per oracle pass, the same for the cpu_baseline leg and the reference arm
@@ -714,7 +728,7 @@ def main():
         "value_two_streams": None if two_stream_ms is None else tokens / (two_stream_ms * 1e-3),
         # FP8: + quantisation of x and of h; ep: route 3, dispatch 5, pack 1, receiver layout 4 + tile prefix 1 + 2 GEMMs +
         # combine 1, finish 1
-        "gpu_launches": (18 if ep_rank is not None else KERNELS_PER_STEP + (2 if fp8 else 0)) * args.steps,
+        "gpu_launches": (18 if ep_rank is not None else kernels_per_step(cfg, args.layer_flags, fp8)) * args.steps,
         "roofline": {"kernel": "ffn_gemm1_kernel (GEMM-1 + SwiGLU, tcgen05)", "bound": "tensor",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": (achieved / peak) if achieved else None,

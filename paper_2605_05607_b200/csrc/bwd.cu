@@ -191,7 +191,7 @@ cudaError_t launch_layer_backward(const Shape& s, const BwdArgs& a, cudaStream_t
     if ((err = ffn::launch_bwd_glu(r, m_w1, m_w3, m_xs, st)) != cudaSuccess) return err;
   }
   // dW2[e] = H^T . dO
-  if ((err = ffn::launch_wgrad(r_h, r_do, a.poff, a.dw2, s.E, s.f, s.d, a.status, st)) != cudaSuccess) return err;
+  if ((err = ffn::launch_wgrad_pair(r_h, r_do, a.poff, a.dw2, s.E, s.f, s.d, a.status, st)) != cudaSuccess) return err;
   // dXs = dA1 . W1^T + dA3 . W3^T : [R, f] x [f, d], twice into one accumulator
   ffn::GemmParams q{};
   q.out = static_cast<__nv_bfloat16*>(a.dxs);
@@ -216,8 +216,8 @@ cudaError_t launch_layer_backward(const Shape& s, const BwdArgs& a, cudaStream_t
   if ((err = launch_combine_rows(sc, a.dxs, Lp, a.topk_idx, nullptr, nullptr, a.dx, (int)R, a.status, st)) != cudaSuccess)
     return err;
   // dW1[e] = Xs^T . dA1,  dW3[e] = Xs^T . dA3
-  if ((err = ffn::launch_wgrad(r_xs, r_da1, a.poff, a.dw1, s.E, s.d, s.f, a.status, st)) != cudaSuccess) return err;
-  return ffn::launch_wgrad(r_xs, r_da3, a.poff, a.dw3, s.E, s.d, s.f, a.status, st);
+  if ((err = ffn::launch_wgrad_pair(r_xs, r_da1, a.poff, a.dw1, s.E, s.d, s.f, a.status, st)) != cudaSuccess) return err;
+  return ffn::launch_wgrad_pair(r_xs, r_da3, a.poff, a.dw3, s.E, s.d, s.f, a.status, st);
 }
 
 }  // namespace tcmoe

@@ -47,6 +47,7 @@ struct GemmParams {
 
 struct Tile {
   int e, n0, row0, rows;
+  int out_row0, kb;   // weight-gradient tiles of the pair kernel: first output row of this CTA, k-blocks of the task
 };
 
 // Task w -> (expert, m-group, n-tile, m-tile in group): expert-major; inside an expert the m-tiles
@@ -76,6 +77,8 @@ __device__ __forceinline__ Tile decode_tile(int w, const int* tp, const int* eof
   t.n0 = (local / gsize) * bn_out;
   t.row0 = eoff[lo] + (g * mg + local % gsize) * rows_per_tile + rank * BM;
   t.rows = min(BM, eoff[lo + 1] - t.row0);
+  t.out_row0 = t.row0;
+  t.kb = 0;
   return t;
 }
 
@@ -154,8 +157,8 @@ bool make_weight_map_fp8(CUtensorMap* map, const void* base, int E, int N, int K
 bool make_act_map_fp8(CUtensorMap* map, const void* base, int rows, int K);
 bool make_weight_map_kmajor(CUtensorMap* map, const void* base, int E, int rows, int cols);
 bool make_rows_map_mn(CUtensorMap* map, const void* base, long long rows, int cols);
-cudaError_t launch_wgrad(const CUtensorMap& m_a, const CUtensorMap& m_b, const int32_t* poff, void* dw, int E, int M,
-                         int N, int32_t* status, cudaStream_t st);
+cudaError_t launch_wgrad_pair(const CUtensorMap& m_a, const CUtensorMap& m_b, const int32_t* poff, void* dw, int E, int M,
+                              int N, int32_t* status, cudaStream_t st);
 
 // fp8 = false: bf16 operands, weights [E, K, N] (B MN-major).  fp8 = true: E4M3 operands, weights
 // [E, N, K] (B K-major), 128 elements of K per pipeline stage, scales applied in the epilogue.

@@ -46,6 +46,7 @@ constexpr int THREADS = 192;
 constexpr uint32_t IDESC = idesc_bf16(2 * BM);
 constexpr uint32_t IDESC_F8 = idesc_e4m3(2 * BM);
 constexpr uint32_t IDESC_BK = idesc_bf16(2 * BM) & ~(1u << 16);   // bf16 with a K-major B operand
+constexpr uint32_t IDESC_WG = idesc_bf16(2 * BM) | (1u << 15);    // bf16 with both operands MN-major
 constexpr uint32_t HINT = 4000;   // try_wait suspend-time hint (ns), see ptx::mbar_try_wait
 
 // RED = false: rows go to o (bf16), Combine is a later pass.  RED = true: Combine happens here
@@ -61,11 +62,16 @@ constexpr uint32_t HINT = 4000;   // try_wait suspend-time hint (ns), see ptx::m
 //                 columns per tile
 //   PAIR_GLU_BWD  the same GEMM recomputed in the backward pass: from a1 = a.W1, a3 = a.W3 and the incoming dh tile the
 //                 epilogue writes h, da1 = dh * a3 * silu'(a1) and da3 = dh * silu(a1)
+//   PAIR_WGRAD    dW[e] = A_e^T . B_e over the rows of expert e in the padded row space (segments start at poff[e], a multiple of 64, pad
+//                 rows zero, so no block of 64 rows mixes experts and an expert without rows gets zeros): a task is a
+//                 256 x 256 tile of one expert's gradient (p.K = its row count M, p.N its columns), the K walk runs over
+//                 the expert's rows in blocks of 64, both operands are MN-major boxes of 64 columns x 64 rows; CTA `rank`
+//                 holds rows m0 + 128 * rank of the tile and columns n0 + 128 * rank of B
 //   PAIR_KSPLIT   acc = A0 . B0 + A1 . B1 (dX = dA1 . W1^T + dA3 . W3^T): the first p.k_split k-blocks come from
 //                 (map_h, map_b0), the rest from (map_a1, map_b1); plain epilogue
 // BKMAJ: the bf16 weight operand is read K-major (one box of 128 columns x 64 K per CTA and stage), which is how
 // W^T looks when W is stored [K, N] with N contiguous: the backward GEMMs read the forward weights in place.
-enum { PAIR_PLAIN = 0, PAIR_GLU = 1, PAIR_GLU_BWD = 2, PAIR_KSPLIT = 3 };
+enum { PAIR_PLAIN = 0, PAIR_GLU = 1, PAIR_GLU_BWD = 2, PAIR_KSPLIT = 3, PAIR_WGRAD = 4 };
 
 template <bool RED, bool FP8, int MODE, bool BKMAJ>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
@@ -129,7 +135,9 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
   ptx::cluster_sync();   // the peer's barriers are initialised before anything signals them
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int total = tp_s[p.E] * p.n_tiles;
+  constexpr bool WGRAD = MODE == PAIR_WGRAD;
+  const int wg_mt = (p.K + 2 * BM - 1) / (2 * BM), wg_per_expert = wg_mt * p.n_tiles;   // weight-gradient tiles per expert
+  const int total = WGRAD ? p.E * wg_per_expert : tp_s[p.E] * p.n_tiles;
   constexpr int BK_ELEMS = FP8 ? 2 * BK : BK;   // K elements per stage: 128 bytes per row either way
   const int KB = MODE == PAIR_KSPLIT ? 2 * p.k_split : (p.K + BK_ELEMS - 1) / BK_ELEMS;
   volatile int* abort_flag = abort_s;
@@ -140,7 +148,21 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
     p.status[ST_ABORT] = 1;
     *abort_flag = 1;
   };
-  auto tile_of = [&](int w) { return decode_tile(w, tp_s, eoff_s, p.E, p.n_tiles, BN_OUT, 2 * BM, rank); };
+  auto tile_of = [&](int w) {
+    if (WGRAD) {   // (expert, m-tile of 256, n-tile of 256), m-tile fastest: neighbours share the B rows in L2
+      Tile t;
+      t.e = w / wg_per_expert;
+      const int rem = w - t.e * wg_per_expert;
+      const int m0 = (rem % wg_mt) * 2 * BM + rank * BM;
+      t.n0 = (rem / wg_mt) * BN_OUT;
+      t.row0 = eoff_s[t.e];                                  // first (padded) row of the expert: start of the K walk
+      t.kb = (eoff_s[t.e + 1] - t.row0) / BK;
+      t.rows = min(BM, p.K - m0);                            // rows of dW[e] this CTA owns (<= 0: none)
+      t.out_row0 = t.e * p.K + m0;
+      return t;
+    }
+    return decode_tile(w, tp_s, eoff_s, p.E, p.n_tiles, BN_OUT, 2 * BM, rank);
+  };
 
   if (warp < 4) {
     // ================================ epilogue (both CTAs) ================================
@@ -156,7 +178,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
       const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * UMMA_N);
       float* yrow = nullptr;
       float wr = 1.f;
-      if (valid && !GLU && (RED || p.topk_w != nullptr)) {
+      if (valid && !GLU && !WGRAD && (RED || p.topk_w != nullptr)) {
         const int pair = __ldg(p.row_pair + grow);
         if (p.topk_w != nullptr) wr = __ldg(p.topk_w + pair);
         if (FP8) wr *= __ldg(p.a_scale + grow);   // row scale of h joins the gate weight
@@ -297,6 +319,10 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
           ptx::tmem_ld32(taddr + cc * 64 + 32, acc1);
           ptx::tmem_ld_wait_on(acc0);
           ptx::tmem_ld_wait_on(acc1);
+          if (WGRAD && t.kb == 0) {   // an expert without rows: the accumulator was never written
+#pragma unroll
+            for (int j = 0; j < 32; ++j) { acc0[j] = 0u; acc1[j] = 0u; }
+          }
           if (FP8) {   // per-output-column weight scales
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -326,7 +352,7 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
               const int r = i * 4 + srow;           // row of this warp's 32
               if (warp * 32 + r < t.rows) {
                 const uint4 q = ptx::ld_shared_v4(stage + r * 144 + piece * 16);
-                *reinterpret_cast<uint4*>(p.out + (size_t)(t.row0 + warp * 32 + r) * (size_t)p.out_ld + col) = q;
+                *reinterpret_cast<uint4*>(p.out + (size_t)(t.out_row0 + warp * 32 + r) * (size_t)p.out_ld + col) = q;
               }
             }
           }
@@ -348,7 +374,8 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
       for (int w = cluster_id; w < total && !*abort_flag; w += num_clusters) {
         const Tile t = tile_of(w);
         bool ok = true;
-        for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int KBt = WGRAD ? t.kb : KB;
+        for (int kb = 0; kb < KBt; ++kb, ++it) {
           const int s = it % NSTAGE;
           if (!ptx::mbar_wait<false, HINT>(empty_bar(s), ((it / NSTAGE) & 1) ^ 1, abort_flag, global_abort)) {
             timeout(2); ok = false; break;
@@ -357,6 +384,14 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
           const uint32_t lead_full = ptx::mapa(full_bar(s), 0);
           // the leader announces the bytes of both CTAs; the peer's copies only complete them
           if (rank == 0) ptx::mbar_arrive_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+          if (WGRAD) {   // four MN-major boxes of 64 columns x 64 rows: this CTA's 128 rows of A^T and 128 columns of B
+            const int r0 = t.row0 + kb * BK, ma = t.out_row0 - t.e * p.K;
+            ptx::tma_load_2d_pair(sa, &map_h, lead_full, ma, r0);
+            ptx::tma_load_2d_pair(sa + 8192, &map_h, lead_full, ma + 64, r0);
+            ptx::tma_load_2d_pair(sb, &map_b0, lead_full, t.n0 + rank * 128, r0);
+            ptx::tma_load_2d_pair(sb + 8192, &map_b0, lead_full, t.n0 + rank * 128 + 64, r0);
+            continue;
+          }
           const bool second = MODE == PAIR_KSPLIT && kb >= p.k_split;     // second (A, B) pair of the K walk
           const int k0 = (second ? kb - p.k_split : kb) * BK_ELEMS;
           ptx::tma_load_2d_pair(sa, second ? &map_a1 : &map_h, lead_full, k0, t.row0);
@@ -387,17 +422,20 @@ ffn_gemm2_kernel(const __grid_constant__ CUtensorMap map_b0, const __grid_consta
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * UMMA_N);
         bool ok = true;
-        for (int kb = 0; kb < KB; ++kb, ++it) {
+        const int KBt = WGRAD ? tile_of(w).kb : KB;
+        for (int kb = 0; kb < KBt; ++kb, ++it) {
           const int s = it % NSTAGE;
           if (!ptx::mbar_wait_cluster<HINT>(full_bar(s), (it / NSTAGE) & 1, abort_flag, global_abort)) {
             timeout(4); ok = false; break;
           }
           ptx::tc_fence_after();
           const uint32_t sa = smem_base + s * STAGE_BYTES, sb = sa + A_BYTES;
-          const uint64_t ad = desc_at(a_base, sa), bd = desc_at(b_base, sb);
+          const uint64_t ad = desc_at(WGRAD ? b_base : a_base, sa), bd = desc_at(b_base, sb);   // WGRAD: A is MN-major too
+          auto bd_a = [](uint64_t d, int k) { return d + (uint64_t)(k * 128); };               // 16 rows of K = 2 KiB
 #pragma unroll
           for (int k = 0; k < 4; ++k) {   // 32 bytes of K per UMMA (16 bf16 / 32 E4M3): +32 B inside the swizzle row
             if (FP8) ptx::umma_f8_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), IDESC_F8, (kb | k) != 0);
+            else if (WGRAD) ptx::umma_bf16_pair(d_tmem, bd_a(ad, k), bd + (uint64_t)(k * 128), IDESC_WG, (kb | k) != 0);
             else if (BKMAJ) ptx::umma_bf16_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 2), IDESC_BK, (kb | k) != 0);
             else ptx::umma_bf16_pair(d_tmem, ad + (uint64_t)(k * 2), bd + (uint64_t)(k * 128), IDESC, (kb | k) != 0);   // B: +2 atoms
           }
@@ -470,6 +508,7 @@ cudaError_t set_pair_attributes() {
     if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, PAIR_PLAIN, true>, attr, SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, PAIR_GLU_BWD, false>, attr, SMEM_BYTES);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, PAIR_KSPLIT, true>, attr, SMEM_BYTES);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(ffn_gemm2_kernel<false, false, PAIR_WGRAD, false>, attr, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_set[dev].store(true, std::memory_order_release);
   }
@@ -526,6 +565,27 @@ cudaError_t launch_bwd_dx(const GemmParams& p, const CUtensorMap& m_w1t, const C
   if (e != cudaSuccess) return e;
   return launch_pdl(ffn_gemm2_kernel<false, false, PAIR_KSPLIT, true>, pair_grid(), THREADS, SMEM_BYTES, st, m_w1t, m_w3t,
                     m_da1, m_da3, p);
+}
+
+// Weight gradient on CTA pairs: dw[e] = A_e^T . B_e, A = [rows, M], B = [rows, N] in the padded row space (maps with
+// boxes of 64 columns x 64 rows), dw [E, M, N] bf16, fully written.
+cudaError_t launch_wgrad_pair(const CUtensorMap& m_a, const CUtensorMap& m_b, const int32_t* poff, void* dw, int E, int M,
+                              int N, int32_t* status, cudaStream_t st) {
+  cudaError_t e = set_pair_attributes();
+  if (e != cudaSuccess) return e;
+  GemmParams p{};
+  p.out = static_cast<__nv_bfloat16*>(dw);
+  p.out_ld = N;
+  p.expert_offsets = poff;
+  p.tile_prefix = poff;      // not used by this mode (the table load needs a valid array)
+  p.E = E;
+  p.K = M;                   // rows of dw[e]
+  p.N = N;
+  p.n_tiles = (N + 255) / 256;
+  p.status = status;
+  ProfileScope prof(KID_WGRAD, st);
+  return launch_pdl(ffn_gemm2_kernel<false, false, PAIR_WGRAD, false>, pair_grid(), THREADS, SMEM_BYTES, st, m_b, m_b, m_a,
+                    m_a, p);
 }
 
 }  // namespace ffn
