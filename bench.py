@@ -400,6 +400,38 @@ def backward_leg(cfg, t, reps=5):
             "routing": "fixed (expert indices and gate weights of the forward; the gate's own gradient is outside)"}
 
 
+def library_context_leg(cfg, t):
+    """Context, not the product: cuBLAS (through torch.bmm) on a BALANCED copy of GEMM-1's problem, on the same
+    weights: E batches of [T k / E, d] x [d, f] with W1 only; no gather, no ragged tiles, no SwiGLU epilogue.  Timed once
+    after idle (burst) and in a loop of about a second (at the board's power limit).  This is the rate the library
+    reaches on this shape and box; the kernel's own fraction is printed against the measured peaks as before."""
+    import time as _time
+    E, d, f = cfg.E, cfg.d, cfg.f
+    R = max(1, cfg.P // E)
+    xs = torch.randn(E, R, d, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    w1 = t["w1"].view(E, d, f)
+    o = torch.empty(E, R, f, device="cuda", dtype=torch.bfloat16)
+    flops = 2.0 * E * R * d * f
+
+    def timed(n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            torch.bmm(xs, w1, out=o)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    timed(3)
+    _time.sleep(0.5)
+    burst = timed(1)
+    n = max(3, int(1000.0 / max(burst, 1e-3)))
+    timed(n // 2)
+    sus = timed(n)
+    return {"what": "torch.bmm (cuBLAS) on E x [T k / E, d] x [d, f], W1 only, balanced rows", "E": E, "rows": R,
+            "tflops_burst": flops / burst / 1e9, "tflops_at_power_limit": flops / sus / 1e9, "loop_calls": n}
+
+
 def workload_config(cfg, n_gpus):
     return {"workload": f"{cfg.name}: T={cfg.T} d={cfg.d} f={cfg.f} E={cfg.E} top-{cfg.k} G={cfg.G} per GPU",
             "T": cfg.T, "d": cfg.d, "f": cfg.f, "E": cfg.E, "k": cfg.k, "G": cfg.G,
@@ -777,6 +809,8 @@ def main():
                                                                       "fused_ms", "unfused_sum_ms")}
     if world == 1 and not args.lean and ep_rank is None and not fp8 and not args.no_backward:
         line["backward"] = backward_leg(cfg, t)
+    if world == 1 and not args.lean and ep_rank is None and not fp8:
+        line["library_context"] = library_context_leg(cfg, t)
     if world == 1 and args.report and not args.lean:
         report = {cfg.name: line["stages"]}
         del t
