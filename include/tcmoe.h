@@ -393,6 +393,14 @@ int moe_payload_efficiency(int64_t transfer_bytes, int32_t n_targets, double out
 enum { MOE_KERNEL_SELFTEST = 9 };
 int moe_selftest_wait_timeout(void* ws, uint64_t limit_ns, void* stream);
 
+/* TMA descriptors.  The tcgen05 kernels read their operands through TMA tensor maps, which are a function of an
+ * operand's address, extents and strides only (not of its contents).  The library keeps the 64 most recent maps,
+ * keyed by every argument of the encode, so that a layer called again on the same weights and workspace does not
+ * encode them again; a buffer freed and reallocated at the same address with the same shape gets the same (still
+ * correct) map.  moe_clear_cache forgets them all (host memory only; nothing on the device).  Thread-safe.
+ * Returns MOE_OK. */
+int moe_clear_cache(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -45,7 +45,7 @@ EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "m
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",
            "moe_profile_enable", "moe_profile_read", "moe_dispatch_noalloc", "moe_quantize_rows",
            "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8", "moe_layer_fp8_host", "moe_selftest_wait_timeout", "moe_traffic_stats", "moe_ep_pack", "moe_ep_finish",
-           "moe_payload_efficiency", "moe_backward_workspace_bytes", "moe_layer_backward")
+           "moe_payload_efficiency", "moe_backward_workspace_bytes", "moe_layer_backward", "moe_clear_cache")
 
 
 class MoEShape(ctypes.Structure):
@@ -334,6 +334,11 @@ KERNEL_IDS = {"topk": 1, "masks": 2, "fill": 3, "dispatch": 4, "gemm1": 5, "gemm
 
 def moe_profile_enable(kernel_id: int) -> None:
     _check("moe_profile_enable", lib().moe_profile_enable(kernel_id))
+
+
+def moe_clear_cache() -> None:
+    """Forget the cached TMA tensor maps (host memory only)."""
+    _check("moe_clear_cache", lib().moe_clear_cache())
 
 
 def moe_profile_read():

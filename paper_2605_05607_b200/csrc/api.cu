@@ -309,6 +309,11 @@ int moe_profile_enable(int kernel_id) {
   return MOE_OK;
 }
 
+int moe_clear_cache(void) {
+  tcmoe::ffn::clear_map_cache();
+  return MOE_OK;
+}
+
 int moe_profile_read(float* total_ms, int32_t* launches) {
   if (total_ms == nullptr || launches == nullptr) return MOE_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_profile_mutex);

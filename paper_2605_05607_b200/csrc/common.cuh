@@ -150,6 +150,9 @@ struct FfnArgs {
 };
 size_t fused_table_blocks(const Shape& s);   // task-block capacity for a shape (ffn_fused.cu)
 size_t fused_tracker_bytes(const Shape& s);  // bytes of the tracker tables for a shape
+namespace ffn {
+void clear_map_cache();                      // forget the cached TMA tensor maps (ffn.cu)
+}
 cudaError_t launch_expert_ffn(const Shape& s, const FfnArgs& a, cudaStream_t st);
 // FP8 form of the expert FFN: a.a_src / a.w1 / a.w3 / a.w2 hold E4M3 codes (weights [E, N, K]).
 struct Fp8Args {

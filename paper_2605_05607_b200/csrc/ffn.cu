@@ -3,9 +3,12 @@
 #include "ffn_common.cuh"
 
 #include <atomic>
+#include <mutex>
 
 namespace tcmoe {
 namespace ffn {
+
+namespace {
 
 EncodeTiledFn encode_fn() {
   static std::atomic<EncodeTiledFn> cached{nullptr};   // looked up once; a second lookup gives the same address
@@ -22,83 +25,115 @@ EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 weights [E, K, N] row-major: box = 64 (N) x 64 (K) x 1, 128-byte swizzle, zero fill
-bool make_weight_map(CUtensorMap* map, const void* base, int E, int K, int N) {
+// A tensor map is a pure function of (address, element size, rank, extents, strides, box): the same arguments give
+// the same 128 bytes, whatever the memory holds.  The layer asks for the same handful of maps on every call (weights,
+// workspace regions), so the most recent ones are kept, keyed by exactly those arguments.
+struct MapKey {
+  const void* base;
+  int bytes, rank;
+  cuuint64_t dims[3], strides[2];
+  cuuint32_t box[3];
+  bool operator==(const MapKey& o) const {
+    return base == o.base && bytes == o.bytes && rank == o.rank && dims[0] == o.dims[0] && dims[1] == o.dims[1] &&
+           dims[2] == o.dims[2] && strides[0] == o.strides[0] && strides[1] == o.strides[1] && box[0] == o.box[0] &&
+           box[1] == o.box[1] && box[2] == o.box[2];
+  }
+};
+struct MapEntry {
+  MapKey key;
+  CUtensorMap map;
+};
+constexpr int MAP_CACHE_ENTRIES = 64;
+std::mutex g_map_mutex;
+MapEntry g_map_cache[MAP_CACHE_ENTRIES];
+int g_map_count = 0, g_map_next = 0;   // entries in use, next slot to overwrite (round robin)
+
+}  // namespace
+
+// Every map of this library: bf16 (bytes = 0) or one-byte (bytes = 1) elements, 128-byte swizzle, no interleave,
+// 256-byte L2 promotion, zero fill outside the tensor.
+bool encode_tiled(CUtensorMap* map, bool bytes, int rank, const void* base, const cuuint64_t* dims,
+                  const cuuint64_t* strides, const cuuint32_t* box) {
+  MapKey key{};
+  key.base = base;
+  key.bytes = bytes ? 1 : 0;
+  key.rank = rank;
+  for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+  for (int i = 0; i + 1 < rank; ++i) key.strides[i] = strides[i];
+  {
+    std::lock_guard<std::mutex> lock(g_map_mutex);
+    for (int i = 0; i < g_map_count; ++i)
+      if (g_map_cache[i].key == key) { *map = g_map_cache[i].map; return true; }
+  }
   EncodeTiledFn fn = encode_fn();
   if (fn == nullptr) return false;
+  const cuuint32_t estr[3] = {1, 1, 1};
+  if (fn(map, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank,
+         const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+         CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  std::lock_guard<std::mutex> lock(g_map_mutex);
+  MapEntry& e = g_map_cache[g_map_next];
+  e.key = key;
+  e.map = *map;
+  g_map_next = (g_map_next + 1) % MAP_CACHE_ENTRIES;
+  if (g_map_count < MAP_CACHE_ENTRIES) ++g_map_count;
+  return true;
+}
+
+void clear_map_cache() {
+  std::lock_guard<std::mutex> lock(g_map_mutex);
+  g_map_count = 0;
+  g_map_next = 0;
+}
+
+// bf16 weights [E, K, N] row-major: box = 64 (N) x 64 (K) x 1, 128-byte swizzle, zero fill
+bool make_weight_map(CUtensorMap* map, const void* base, int E, int K, int N) {
   cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)K, (cuuint64_t)E};
   cuuint64_t strides[2] = {(cuuint64_t)N * 2, (cuuint64_t)N * K * 2};
   cuuint32_t box[3] = {64, BK, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled(map, false, 3, base, dims, strides, box);
 }
 
 // bf16 activations [rows, K] row-major: box = 64 (K) x 128 rows
 bool make_act_map(CUtensorMap* map, const void* base, long long rows, int K) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return false;
   cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)K * 2};
   cuuint32_t box[2] = {BK, BM};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled(map, false, 2, base, dims, strides, box);
 }
 
 // E4M3 weights [E, N, K] (K contiguous): box = 128 bytes of K x 128 output columns x 1, 128-byte swizzle
 bool make_weight_map_fp8(CUtensorMap* map, const void* base, int E, int N, int K) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return false;
   cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)N, (cuuint64_t)E};
   cuuint64_t strides[2] = {(cuuint64_t)K, (cuuint64_t)N * K};
   cuuint32_t box[3] = {128, 128, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled(map, true, 3, base, dims, strides, box);
 }
 
 // E4M3 activations [rows, K]: box = 128 bytes of K x 128 rows
 bool make_act_map_fp8(CUtensorMap* map, const void* base, int rows, int K) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return false;
   cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)K};
   cuuint32_t box[2] = {128, BM};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled(map, true, 2, base, dims, strides, box);
 }
 
 // bf16 weights [E, K, N] read as the TRANSPOSED operand of a backward GEMM: the same memory seen as [E, N' = K, K' = N]
 // with K' contiguous; box = 64 (K') x 128 (N') x 1, 128-byte swizzle.  `rows` = N', `cols` = K'.
 bool make_weight_map_kmajor(CUtensorMap* map, const void* base, int E, int rows, int cols) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return false;
   cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)E};
   cuuint64_t strides[2] = {(cuuint64_t)cols * 2, (cuuint64_t)rows * cols * 2};
   cuuint32_t box[3] = {64, 128, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled(map, false, 3, base, dims, strides, box);
 }
 
 // bf16 rows [rows, cols] read with the row index as K (weight gradients): box = 64 columns x 64 rows
 bool make_rows_map_mn(CUtensorMap* map, const void* base, long long rows, int cols) {
-  EncodeTiledFn fn = encode_fn();
-  if (fn == nullptr) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
   cuuint32_t box[2] = {64, 64};
-  cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_tiled(map, false, 2, base, dims, strides, box);
 }
 
 }  // namespace ffn

@@ -150,7 +150,11 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// tensor maps (ffn.cu)
+// tensor maps (ffn.cu).  encode_tiled is the one place that calls cuTensorMapEncodeTiled; it keeps the most recent maps,
+// keyed by every argument of the encode, and clear_map_cache forgets them.
+bool encode_tiled(CUtensorMap* map, bool bytes, int rank, const void* base, const cuuint64_t* dims,
+                  const cuuint64_t* strides, const cuuint32_t* box);
+void clear_map_cache();
 bool make_weight_map(CUtensorMap* map, const void* base, int E, int K, int N);
 bool make_act_map(CUtensorMap* map, const void* base, long long rows, int K);
 bool make_weight_map_fp8(CUtensorMap* map, const void* base, int E, int N, int K);

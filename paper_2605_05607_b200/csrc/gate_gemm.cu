@@ -219,21 +219,6 @@ gate_umma_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constan
   }
 }
 
-EncodeTiledFn encoder() {
-  static std::atomic<EncodeTiledFn> cached{nullptr};   // looked up once; a second lookup gives the same address
-  EncodeTiledFn fn = cached.load(std::memory_order_acquire);
-  if (fn == nullptr) {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
-        q == cudaDriverEntryPointSuccess) {
-      fn = reinterpret_cast<EncodeTiledFn>(sym);
-      cached.store(fn, std::memory_order_release);
-    }
-  }
-  return fn;
-}
-
 }  // namespace
 
 size_t gate_split_bytes(int d, int E) { return (size_t)3 * d * ((E + 63) & ~63) * 2; }
@@ -250,28 +235,18 @@ cudaError_t launch_gate_logits(const Shape& s, const void* x, const float* w_gat
     attr_set[dev].store(true, std::memory_order_release);
   }
   const int Epad = (s.E + 63) & ~63;
-  EncodeTiledFn fn = encoder();
-  if (fn == nullptr) return cudaErrorInvalidValue;
   CUtensorMap m_x, m_w;
   {
     cuuint64_t dims[2] = {(cuuint64_t)s.d, (cuuint64_t)s.T};
     cuuint64_t strides[1] = {(cuuint64_t)s.d * 2};
     cuuint32_t box[2] = {BK, BM};
-    cuuint32_t estr[2] = {1, 1};
-    if (fn(&m_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), dims, strides, box, estr,
-           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return cudaErrorInvalidValue;
+    if (!ffn::encode_tiled(&m_x, false, 2, x, dims, strides, box)) return cudaErrorInvalidValue;
   }
   {
     cuuint64_t dims[3] = {(cuuint64_t)Epad, (cuuint64_t)s.d, 3};
     cuuint64_t strides[2] = {(cuuint64_t)Epad * 2, (cuuint64_t)Epad * s.d * 2};
     cuuint32_t box[3] = {64, BK, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    if (fn(&m_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, wsplit, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-      return cudaErrorInvalidValue;
+    if (!ffn::encode_tiled(&m_w, false, 3, wsplit, dims, strides, box)) return cudaErrorInvalidValue;
   }
   ProfileScope prof(KID_GATE, st);
   const size_t n = (size_t)s.d * Epad;

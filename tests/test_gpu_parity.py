@@ -529,3 +529,42 @@ def test_pair_gemm1_on_the_per_expert_layout_tensors(cfg):
     o_ref, y_ref = run.o.clone(), run.y.clone()
     _check_single_kernel(cfg, run, B.MOE_FLAG_GEMM1_PAIR, o_ref, y_ref)
     staged(cfg, B.MOE_FLAG_GEMM1_PAIR)
+
+
+def test_tensor_map_cache_is_transparent():
+    """The TMA descriptors are cached by (address, extents, strides, box).  Same inputs through a warm cache, a cleared
+    cache, and a cache that has been flooded by another shape in between must give bit-identical outputs; and a new
+    tensor that lands at a recycled address with another shape must get its own descriptor."""
+    cfg = synth.CONFIGS["C1"]
+    run = H.Run(cfg)
+    run.layer()
+    torch.cuda.synchronize()
+    y0 = H.bf16_host(run.y).copy()
+    run.layer()                       # warm cache
+    torch.cuda.synchronize()
+    assert np.array_equal(H.bf16_host(run.y), y0)
+    B.moe_clear_cache()
+    run.layer()                       # everything encoded again
+    torch.cuda.synchronize()
+    assert np.array_equal(H.bf16_host(run.y), y0)
+    # more distinct maps than the cache holds, some of them at addresses the allocator hands out again
+    for i in range(12):
+        other = H.Run(cfg.with_(name=f"c1_{i}", T=128 + 64 * i, d=256 + 64 * (i % 3), f=512))
+        other.layer()
+        torch.cuda.synchronize()
+        assert other.status()[0] == 0
+        del other
+    run.layer()
+    torch.cuda.synchronize()
+    assert np.array_equal(H.bf16_host(run.y), y0)
+    assert run.status()[0] == 0
+    # the same check against the oracle on a shape that reuses freed memory
+    torch.cuda.empty_cache()
+    cfg2 = cfg.with_(name="c1_small", T=192, d=384, f=768)
+    r2 = H.Run(cfg2)
+    r2.layer(logits=r2.logits)
+    torch.cuda.synchronize()
+    _, _, _, y_def = O.layer(H.bf16_host(r2.t["x"]), r2.host_logits(), r2.host_bias(), H.bf16_host(r2.t["w1"]),
+                             H.bf16_host(r2.t["w3"]), H.bf16_host(r2.t["w2"]), cfg2.k, cfg2.score_fn)
+    H.assert_close_out(O.bf16_to_f64(H.bf16_host(r2.y)[: cfg2.T]), y_def, "layer after cache churn")
+    assert r2.status()[0] == 0
