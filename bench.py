@@ -509,7 +509,7 @@ def main():
     ap.add_argument("--parallel", default="replicas", choices=["replicas", "ep"],
                     help="multi-GPU form: replicas (default: weights replicated, tokens sharded, no data-path "
                          "collective) or ep (expert parallelism: group g on rank g, all-to-all of the dispatched rows "
-                         "and of the pre-reduced rows; needs E % N == 0; bf16 experts)")
+                         "and of the pre-reduced rows; needs E divisible by N; bf16 experts)")
     ap.add_argument("--layer-flags", type=int, default=0,
                     help="MOE_FLAG_* bits for the timed moe_layer call (2: Combine in GEMM-2's epilogue, 8: GEMM-1 + GEMM-2 "
                          "as one tracker-paced kernel, 24: the same with the SM partition); default 0")
@@ -519,6 +519,8 @@ def main():
     ap.add_argument("--lean", action="store_true",
                     help="timed region only: no e2e / stage / cpu_baseline legs (for profiler captures)")
     ap.add_argument("--no-backward", action="store_true", help="skip the backward / training-step leg")
+    ap.add_argument("--with-backward", action="store_true",
+                    help="run the backward / training-step leg even with --lean (for profiler captures of its kernels)")
     ap.add_argument("--stages-only", action="store_true",
                     help="only the per-stage breakdown of --config (prints its JSON); for profiler captures")
     ap.add_argument("--no-ffn", action="store_true", help="with --stages-only: skip expert weights and the FFN")
@@ -807,8 +809,8 @@ def main():
                                                                           "frac_bf16_burst", "frac_bf16_sustained")}
         line["fused_vs_unfused_ms"] = {k: st["summary"][k] for k in ("fused_back_to_back_ms", "unfused_back_to_back_ms",
                                                                       "fused_ms", "unfused_sum_ms")}
-    if world == 1 and not args.lean and ep_rank is None and not fp8 and not args.no_backward:
-        line["backward"] = backward_leg(cfg, t)
+    if world == 1 and (not args.lean or args.with_backward) and ep_rank is None and not fp8 and not args.no_backward:
+        line["backward"] = backward_leg(cfg, t, reps=1 if args.lean else 5)
     if world == 1 and not args.lean and ep_rank is None and not fp8:
         line["library_context"] = library_context_leg(cfg, t)
     if world == 1 and args.report and not args.lean:
