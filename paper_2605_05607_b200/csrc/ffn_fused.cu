@@ -173,7 +173,7 @@ ffn_fused_kernel(const __grid_constant__ CUtensorMap map_w1, const __grid_consta
     p.status[ST_ABORT] = 1;
     *abort_flag = 1;
   };
-  // bounded wait of one warp on a tracker counter (lane 0 polls, all lanes get the verdict)
+  // bounded wait of one warp on a tracker counter (lane 0 polls, all lanes get the result)
   auto wait_counter = [&](const int32_t* ctr, int want, int detail) -> bool {
     int ok = 1;
     if (lane == 0) {
