@@ -338,6 +338,53 @@ def layer_backward(x_bits: np.ndarray, topk_idx: np.ndarray, topk_w: np.ndarray,
     return dx, grads
 
 
+def gate_backward(x_bits: np.ndarray, w_gate: np.ndarray, bias: Optional[np.ndarray], topk_idx: np.ndarray,
+                  score_fn: int, w1_bits, w3_bits, w2_bits, dy: np.ndarray):
+    """Gradient that reaches the gate network when the SELECTION is held fixed but the gate weights are functions of
+    the router keys (Sec. II-A: the gate picks the topk experts and weighs their outputs; Sec. VI-A: training).  With
+        key[t, e] = x[t] . w_gate[:, e] + bias[t, e],   w[t, :] = softmax / renormalised sigmoid of key[t, topk_idx[t, :]],
+        y[t] = sum_j w[t, j] * FFN_{idx[t, j]}(x[t])   and   L = sum(dy * y):
+        dL/dw[t, j]   = dy[t] . FFN_{idx[t, j]}(x[t])
+        dL/dkey[t, j] = softmax:  w_j (dL/dw_j - sum_i w_i dL/dw_i)
+                        sigmoid:  s_j (1 - s_j) (dL/dw_j - sum_i w_i dL/dw_i) / sum_i s_i,   s = sigmoid(key)
+        dL/dw_gate    = x^T . dlogits      (dlogits[t, e] = dL/dkey[t, j] at e = idx[t, j], else 0)
+        dx_gate[t]    = dlogits[t] . w_gate^T          (added to the dx of ``layer_backward``).
+    All in fp64; keys are formed in fp64 from the bf16 x and the fp32 gate weight (no rounding of the logits).
+    Returns (dw_gate [d, E], dx_gate [T, d], dkey [T, k], dL/dw [T, k])."""
+    idx = np.asarray(topk_idx, dtype=np.int64)
+    x = bf16_to_f64(x_bits)
+    wg = np.asarray(w_gate, dtype=np.float32).astype(np.float64)
+    T, k = idx.shape
+    keys = x @ wg
+    if bias is not None:
+        b = np.asarray(bias, dtype=np.float32).astype(np.float64)
+        keys = keys + (b[None, :] if b.ndim == 1 else b)
+    sel = np.take_along_axis(keys, idx, axis=1)
+    if score_fn == SCORE_SOFTMAX:
+        z = np.exp(sel - sel.max(axis=1, keepdims=True))
+        w = z / z.sum(axis=1, keepdims=True)
+    elif score_fn == SCORE_SIGMOID:
+        sg = 1.0 / (1.0 + np.exp(-sel))
+        ssum = sg.sum(axis=1, keepdims=True)
+        w = sg / ssum
+    else:
+        raise ValueError("score_fn must be 0 (softmax) or 1 (sigmoid)")
+    dyf = np.asarray(dy, dtype=np.float64)
+    dw = np.zeros((T, k), dtype=np.float64)
+    for e in np.unique(idx):
+        hit_t, hit_j = np.nonzero(idx == e)
+        o = expert_ffn_rows(x[hit_t], w1_bits[e], w3_bits[e], w2_bits[e])
+        dw[hit_t, hit_j] = np.sum(o * dyf[hit_t], axis=1)
+    centred = dw - np.sum(w * dw, axis=1, keepdims=True)
+    if score_fn == SCORE_SOFTMAX:
+        dkey = w * centred
+    else:
+        dkey = sg * (1.0 - sg) * centred / ssum
+    dlogits = np.zeros_like(keys)
+    np.put_along_axis(dlogits, idx, dkey, axis=1)
+    return x.T @ dlogits, dlogits @ wg.T, dkey, dw
+
+
 # --------------------------------------------------------------------------- traffic counters
 def distinct_groups_per_token(topk_idx: np.ndarray, E: int, G: int) -> float:
     """Mean number D of distinct destination groups per token = N_disp / T."""

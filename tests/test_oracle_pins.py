@@ -579,3 +579,107 @@ def test_layer_backward_is_the_routed_sum_of_expert_gradients():
     # linear in dy
     dx2, grads2 = O.layer_backward(xb, idx, w, w1b, w3b, w2b, 2.0 * dy)
     assert np.array_equal(dx2, 2.0 * dx) and np.array_equal(grads2[0][2], 2.0 * grads[0][2])
+
+
+def _gate_case(rng, score_fn, k=3, with_bias=True):
+    T, d, f, E = 5, 8, 6, 6
+    xb = O.f64_to_bf16_bits(rng.standard_normal((T, d)))
+    wg = (rng.standard_normal((d, E)) * 0.3).astype(np.float32)
+    bias = (rng.standard_normal((T, E)) * 0.2).astype(np.float32) if with_bias else None
+    w1b, w3b, w2b = (O.f64_to_bf16_bits(rng.standard_normal(s) * 0.4) for s in ((E, d, f), (E, d, f), (E, f, d)))
+    idx = np.stack([rng.permutation(E)[:k] for _ in range(T)]).astype(np.int32)     # any fixed selection
+    dy = rng.standard_normal((T, d))
+    return xb, wg, bias, idx, w1b, w3b, w2b, dy, score_fn
+
+
+def _gate_forward_loss(x64, wg64, bias, idx, w1b, w3b, w2b, dy, score_fn):
+    """L = sum(dy * y) through the oracle's own forward pieces (gate_weights and expert_ffn_rows, each pinned above)
+    with the selection fixed; keys in fp64 so that a difference quotient sees the perturbation."""
+    keys = x64 @ wg64 + (0.0 if bias is None else bias.astype(np.float64))
+    sel = np.take_along_axis(keys, idx.astype(np.int64), axis=1)
+    # gate_weights rounds its keys to fp32 first; feed it per-row shifted keys is not possible, so the weights
+    # come from the same definition evaluated by torch in fp64 (softmax / sigmoid are library routines there)
+    ts = torch.tensor(sel, dtype=torch.float64)
+    w = (torch.softmax(ts, dim=1) if score_fn == O.SCORE_SOFTMAX
+         else torch.sigmoid(ts) / torch.sigmoid(ts).sum(dim=1, keepdim=True)).numpy()
+    total = 0.0
+    for t in range(x64.shape[0]):
+        for j in range(idx.shape[1]):
+            e = idx[t, j]
+            o = O.expert_ffn_rows_f64(x64[t:t + 1], O.bf16_to_f64(w1b[e]), O.bf16_to_f64(w3b[e]), O.bf16_to_f64(w2b[e]))[0]
+            total += w[t, j] * float(dy[t] @ o)
+    return total
+
+
+@pytest.mark.parametrize("score_fn", [O.SCORE_SOFTMAX, O.SCORE_SIGMOID])
+def test_gate_backward_against_central_finite_differences(score_fn):
+    """dL/dw_gate (every entry) and the total dL/dx (gate path + expert path) against central differences of the
+    forward with the selection held fixed.  A wrong sign or a dropped renormalisation term in the softmax / sigmoid
+    derivative, a transposed gate weight, or a gate path missing from dx fails it."""
+    xb, wg, bias, idx, w1b, w3b, w2b, dy, _ = _gate_case(np.random.default_rng(11 + score_fn), score_fn)
+    x64, wg64 = O.bf16_to_f64(xb), wg.astype(np.float64)
+    dwg, dxg, dkey, dw = O.gate_backward(xb, wg, bias, idx, score_fn, w1b, w3b, w2b, dy)
+    # the weights the expert path of dx needs: the oracle's own gate_weights on the fp32 keys
+    keys32 = (x64 @ wg64 + bias.astype(np.float64)).astype(np.float32)
+    w = O.gate_weights(keys32, idx, score_fn)
+    dx_exp, _ = O.layer_backward(xb, idx, w, w1b, w3b, w2b, dy)
+    loss = lambda x_, wg_: _gate_forward_loss(x_, wg_, bias, idx, w1b, w3b, w2b, dy, score_fn)
+    eps = 1e-6
+    num = np.zeros_like(wg64)
+    for i in np.ndindex(wg64.shape):
+        hi, lo = wg64.copy(), wg64.copy()
+        hi[i] += eps
+        lo[i] -= eps
+        num[i] = (loss(x64, hi) - loss(x64, lo)) / (2 * eps)
+    assert np.abs(num - dwg).max() <= 1e-6 * max(1.0, np.abs(dwg).max())
+    numx = np.zeros_like(x64)
+    for i in np.ndindex(x64.shape):
+        hi, lo = x64.copy(), x64.copy()
+        hi[i] += eps
+        lo[i] -= eps
+        numx[i] = (loss(hi, wg64) - loss(lo, wg64)) / (2 * eps)
+    # gate_weights saw fp32-rounded keys: the expert path carries that 1e-7 relative difference
+    assert np.abs(numx - (dx_exp + dxg)).max() <= 1e-5 * max(1.0, np.abs(numx).max())
+    assert np.abs(dxg).max() > 1e-3 * np.abs(numx).max()          # the gate path is not negligible in this case
+
+
+@pytest.mark.parametrize("score_fn", [O.SCORE_SOFTMAX, O.SCORE_SIGMOID])
+def test_gate_backward_against_fp64_autograd(score_fn):
+    """The same quantities from torch's fp64 automatic differentiation of a dense re-statement of the layer
+    (gather of the selected keys, library softmax / sigmoid, matmul experts)."""
+    xb, wg, bias, idx, w1b, w3b, w2b, dy, _ = _gate_case(np.random.default_rng(21 + score_fn), score_fn)
+    tx = torch.tensor(O.bf16_to_f64(xb), requires_grad=True)
+    tg = torch.tensor(wg.astype(np.float64), requires_grad=True)
+    keys = tx @ tg + torch.tensor(bias.astype(np.float64))
+    sel = torch.gather(keys, 1, torch.tensor(idx.astype(np.int64)))
+    w = torch.softmax(sel, 1) if score_fn == O.SCORE_SOFTMAX else torch.sigmoid(sel) / torch.sigmoid(sel).sum(1, keepdim=True)
+    w_const = w.detach()
+    y_gate = torch.zeros(tx.shape, dtype=torch.float64)      # gradient flows through the weights only
+    y_exp = torch.zeros(tx.shape, dtype=torch.float64)       # gradient flows through the experts only
+    for t in range(tx.shape[0]):
+        for j in range(idx.shape[1]):
+            e = int(idx[t, j])
+            t1, t3, t2 = (torch.tensor(O.bf16_to_f64(v[e])) for v in (w1b, w3b, w2b))
+            ffn = lambda a: (torch.nn.functional.silu(a @ t1) * (a @ t3)) @ t2
+            y_gate[t] = y_gate[t] + w[t, j] * ffn(tx[t:t + 1].detach())[0]
+            y_exp[t] = y_exp[t] + w_const[t, j] * ffn(tx[t:t + 1])[0]
+    tdy = torch.tensor(dy)
+    gwg, gx_gate = torch.autograd.grad((y_gate * tdy).sum(), (tg, tx), retain_graph=True)
+    dwg, dxg, dkey, dw = O.gate_backward(xb, wg, bias, idx, score_fn, w1b, w3b, w2b, dy)
+    assert np.abs(dwg - gwg.numpy()).max() <= 1e-12 * max(1.0, np.abs(dwg).max())
+    assert np.abs(dxg - gx_gate.numpy()).max() <= 1e-12 * max(1.0, np.abs(dxg).max())
+
+
+def test_gate_backward_special_cases():
+    """k = 1: the single weight is 1 whatever the key, so nothing reaches the gate.  Softmax: shifting every selected
+    key of a token leaves its weights unchanged, so the key gradients of a token sum to zero.  The gate path is linear
+    in dy."""
+    for score_fn in (O.SCORE_SOFTMAX, O.SCORE_SIGMOID):
+        xb, wg, bias, idx, w1b, w3b, w2b, dy, _ = _gate_case(np.random.default_rng(31), score_fn, k=1)
+        dwg, dxg, dkey, dw = O.gate_backward(xb, wg, bias, idx, score_fn, w1b, w3b, w2b, dy)
+        assert np.abs(dwg).max() <= 1e-15 and np.abs(dxg).max() <= 1e-15 and np.abs(dw).max() > 0.1
+    xb, wg, bias, idx, w1b, w3b, w2b, dy, _ = _gate_case(np.random.default_rng(32), O.SCORE_SOFTMAX, k=4, with_bias=False)
+    dwg, dxg, dkey, dw = O.gate_backward(xb, wg, bias, idx, O.SCORE_SOFTMAX, w1b, w3b, w2b, dy)
+    assert np.abs(dkey.sum(axis=1)).max() <= 1e-14 * np.abs(dkey).max()
+    dwg2, dxg2, _, _ = O.gate_backward(xb, wg, bias, idx, O.SCORE_SOFTMAX, w1b, w3b, w2b, 3.0 * dy)
+    assert np.allclose(dwg2, 3.0 * dwg, rtol=1e-13, atol=0) and np.allclose(dxg2, 3.0 * dxg, rtol=1e-13, atol=0)
