@@ -355,9 +355,9 @@ def stage_breakdown(cfg, t, reps=5, with_ffn=True):
 
 
 def backward_leg(cfg, t, reps=5):
-    """moe_layer_backward (fixed routing from the forward) on the same workload: device time per call, and the
-    training step (forward + backward) it gives.  Useful flops: 12 P d f of gradient GEMMs + 4 P d f of GEMM-1
-    recomputed for its pre-activations."""
+    """moe_layer_backward + moe_gate_backward (the selection of the forward held fixed) on the same workload: device
+    time per call, and the training step (forward + backward) it gives.  Useful flops: 12 P d f of gradient GEMMs +
+    4 P d f of GEMM-1 recomputed for its pre-activations (the gate's gradient adds no GEMM)."""
     from paper_2605_05607_b200 import binding as B
     shape = B.make_shape(cfg)
     ws = B.alloc_workspace(shape)
@@ -371,13 +371,16 @@ def backward_leg(cfg, t, reps=5):
     dx = torch.empty_like(y)
     dw1, dw3, dw2 = torch.empty_like(t["w1"]), torch.empty_like(t["w3"]), torch.empty_like(t["w2"])
     bws = torch.zeros(B.moe_backward_workspace_bytes(shape), dtype=torch.uint8, device=dev)
+    logits = torch.zeros(T * E, dtype=torch.float32, device=dev)
+    dwg = torch.empty(d, E, dtype=torch.float32, device=dev)
 
     def fwd():
-        B.moe_layer(shape, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws, topk_idx=idx, topk_w=w,
-                    layout=lay)
+        B.moe_layer(shape, t["x"], t["w_gate"], t["bias"], t["w1"], t["w3"], t["w2"], y, ws, logits=logits,
+                    topk_idx=idx, topk_w=w, layout=lay)
 
     def bwd():
         B.moe_layer_backward(shape, t["x"], dy, idx, w, lay, t["w1"], t["w3"], t["w2"], dx, dw1, dw3, dw2, bws)
+        B.moe_gate_backward(shape, logits, t["bias"], idx, w, lay, t["w_gate"], dx, dwg, bws)
 
     def timed(fn, n):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -393,11 +396,18 @@ def backward_leg(cfg, t, reps=5):
     assert B.moe_status(bws)[0] == 0
     f_ms, b_ms = timed(fwd, reps), timed(bwd, reps)
     step_ms = timed(lambda: (fwd(), bwd()), reps)
+    B.moe_profile_enable(B.KERNEL_IDS["gate_bwd"])
+    for _ in range(reps):
+        bwd()
+    gate_ms, gate_n = B.moe_profile_read()
+    B.moe_profile_enable(0)
     assert B.moe_status(bws)[0] == 0 and B.moe_status(ws)[0] == 0
     return {"backward_ms": b_ms, "forward_ms": f_ms, "training_step_ms": step_ms,
             "training_tokens_per_s": T / step_ms * 1e3, "backward_tflops": 16.0 * P * d * f / b_ms / 1e9,
+            "gate_backward_ms": gate_ms / max(gate_n, 1),
             "flops_counted": "12 P d f gradient GEMMs + 4 P d f recomputed GEMM-1", "reps": reps,
-            "routing": "fixed (expert indices and gate weights of the forward; the gate's own gradient is outside)"}
+            "gradients": "dx, dW1, dW3, dW2, dw_gate; the selection (expert indices) of the forward held fixed, the "
+                         "gate weights differentiated through the router keys"}
 
 
 def library_context_leg(cfg, t):

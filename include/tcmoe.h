@@ -237,6 +237,25 @@ int moe_layer_backward(const moe_shape_t* shape, const void* x, const void* dy, 
                        const float* topk_w, const moe_layout_t* layout, const void* w1, const void* w3, const void* w2,
                        void* dx, void* dw1, void* dw3, void* dw2, void* ws, size_t ws_bytes, void* stream);
 
+/* Gradient of the gate network (Sec. II-A: the gate picks the topk experts of a token and weighs their outputs;
+ * Sec. VI-A: training).  The SELECTION (topk_idx) is held fixed; the gate weights are differentiated as functions of
+ * the router keys key[t, e] = x[t] . w_gate[:, e] + logit_bias[t, e] (softmax over the k selected keys, or sigmoid
+ * renormalised over them, as shape->score_fn says).  With g[t, j] = topk_w[t, j] * dy[t] . FFN_{e_j}(x[t]):
+ *     dkey[t, j] = (g[t, j] - topk_w[t, j] * sum_i g[t, i]) * c,   c = 1 (softmax) or 1 - sigmoid(key[t, j]),
+ *     dw_gate[:, e] = sum over the pairs (t, j) with e_j = e of dkey[t, j] * x[t, :]        fp32 [d, E], written whole,
+ *     dx[t, :]     += sum_j dkey[t, j] * w_gate[:, e_j]                                     bf16 [T, d], in / out.
+ * MUST follow moe_layer_backward for the same shape, routing and backward workspace on the same stream: it reads
+ * what that call leaves in `ws` (the recomputed h, dH, the per-expert rows of x and the padded row numbers) and the
+ * dx it wrote.  `logits` are the forward's fp32 router logits [T, E] (moe_layer's optional output); required for
+ * sigmoid scores, ignored (may be NULL) for softmax.  logit_bias / bias_row_stride as in moe_route.  `layout` is the
+ * forward's layout (only expert_counts is read).  shape->flags: 0 or MOE_FLAG_SPARSE_TOPK.
+ * Alignment: dx and ws 128 bytes, the other pointers 16.  Errors as moe_layer_backward; sigmoid scores without
+ * logits: MOE_ERR_INVALID_ARG.  Five small launches; deterministic (each expert's rows are summed in ascending
+ * order, no atomics). */
+int moe_gate_backward(const moe_shape_t* shape, const float* logits, const float* logit_bias, int64_t bias_row_stride,
+                      const int32_t* topk_idx, const float* topk_w, const moe_layout_t* layout, const float* w_gate,
+                      void* dx, float* dw_gate, void* ws, size_t ws_bytes, void* stream);
+
 /* ---- FP8 form of the expert FFN --------------------------------------------------------------
  * Sec. V-A evaluates the DeepSeek-V3 experts with FP8 GEMM kernels and gives no recipe; this
  * library's reading: E4M3 elements (largest finite value 448, round to nearest even, saturating),
@@ -316,7 +335,7 @@ int moe_workspace_layout(const moe_shape_t* shape, size_t out[4]);
 /* Kernel ids for moe_profile_enable (also the `where` slot of moe_status). */
 enum { MOE_KERNEL_TOPK = 1, MOE_KERNEL_MASKS = 2, MOE_KERNEL_FILL = 3, MOE_KERNEL_DISPATCH = 4,
        MOE_KERNEL_GEMM1 = 5, MOE_KERNEL_GEMM2 = 6, MOE_KERNEL_COMBINE = 7, MOE_KERNEL_GATE = 8,
-       MOE_KERNEL_WGRAD = 10, MOE_KERNEL_BWD_GATHER = 11 };
+       MOE_KERNEL_WGRAD = 10, MOE_KERNEL_BWD_GATHER = 11, MOE_KERNEL_GATE_BWD = 12 };
 
 /* Per-kernel timing hook for benchmarks (host-side state, one record per process, guarded by a
  * mutex so that launches from several host threads are safe; not part of the method).  After moe_profile_enable(id) every launch of that kernel by any entry point is

@@ -45,7 +45,7 @@ EXPORTS = ("moe_workspace_bytes", "moe_workspace_layout", "moe_status_reset", "m
            "moe_route", "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host",
            "moe_profile_enable", "moe_profile_read", "moe_dispatch_noalloc", "moe_quantize_rows",
            "moe_quantize_weights", "moe_expert_ffn_fp8", "moe_layer_fp8", "moe_layer_fp8_host", "moe_selftest_wait_timeout", "moe_traffic_stats", "moe_ep_pack", "moe_ep_finish",
-           "moe_payload_efficiency", "moe_backward_workspace_bytes", "moe_layer_backward", "moe_clear_cache")
+           "moe_payload_efficiency", "moe_backward_workspace_bytes", "moe_layer_backward", "moe_clear_cache", "moe_gate_backward")
 
 
 class MoEShape(ctypes.Structure):
@@ -100,6 +100,7 @@ def lib() -> ctypes.CDLL:
         L.moe_payload_efficiency.argtypes = [i64, ctypes.c_int32, ctypes.POINTER(ctypes.c_double)]
         L.moe_backward_workspace_bytes.argtypes = [shp, ctypes.POINTER(sz)]
         L.moe_layer_backward.argtypes = [shp, vp, vp, vp, vp, lay, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.moe_gate_backward.argtypes = [shp, vp, vp, i64, vp, vp, lay, vp, vp, vp, vp, sz, vp]
         L.moe_ep_pack.argtypes = [shp, vp, vp, lay, vp, vp, vp]
         L.moe_ep_finish.argtypes = [shp, vp, lay, vp, vp]
         L.moe_profile_enable.argtypes = [ctypes.c_int]
@@ -301,6 +302,16 @@ def moe_layer_backward(shape, x, dy, topk_idx, topk_w, layout: Layout, w1, w3, w
                                                           ws.numel(), _stream(stream)))
 
 
+def moe_gate_backward(shape, logits, logit_bias, topk_idx, topk_w, layout: Layout, w_gate, dx, dw_gate, ws,
+                      stream=None) -> None:
+    """Gate gradient after moe_layer_backward on the same backward workspace: adds the gate path to dx, writes dw_gate."""
+    stride = 0 if logit_bias is None or logit_bias.dim() == 1 else shape.E
+    c = layout.c()
+    _check("moe_gate_backward", lib().moe_gate_backward(ctypes.byref(shape), _ptr(logits), _ptr(logit_bias), stride,
+                                                        _ptr(topk_idx), _ptr(topk_w), ctypes.byref(c), _ptr(w_gate),
+                                                        _ptr(dx), _ptr(dw_gate), _ptr(ws), ws.numel(), _stream(stream)))
+
+
 def moe_selftest_wait_timeout(ws, limit_ns: int, stream=None) -> None:
     _check("moe_selftest_wait_timeout", lib().moe_selftest_wait_timeout(_ptr(ws), limit_ns, _stream(stream)))
 
@@ -329,7 +340,7 @@ def moe_layer_host(shape, x_host, x_dev, w_gate, logit_bias, w1, w3, w2, y_dev, 
 
 
 KERNEL_IDS = {"topk": 1, "masks": 2, "fill": 3, "dispatch": 4, "gemm1": 5, "gemm2": 6, "combine": 7, "gate": 8,
-              "wgrad": 10, "bwd_gather": 11}
+              "wgrad": 10, "bwd_gather": 11, "gate_bwd": 12}
 
 
 def moe_profile_enable(kernel_id: int) -> None:

@@ -8,7 +8,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libtcmoe.so")
-SOURCES = ["api.cu", "route.cu", "gate_gemm.cu", "layout.cu", "ffn.cu", "ffn_gemm1.cu", "ffn_gemm2.cu", "ffn_fused.cu", "quant.cu", "ep.cu", "noalloc.cu", "bwd.cu"]
+SOURCES = ["api.cu", "route.cu", "gate_gemm.cu", "layout.cu", "ffn.cu", "ffn_gemm1.cu", "ffn_gemm2.cu", "ffn_fused.cu", "quant.cu", "ep.cu", "noalloc.cu", "bwd.cu", "gate_bwd.cu"]
 HEADERS = ["common.cuh", "ptx.cuh", "ffn_common.cuh", "combine.cuh", os.path.join("..", "..", "include", "tcmoe.h")]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-cudart", "static"]

@@ -302,7 +302,7 @@ int moe_selftest_wait_timeout(void* ws, uint64_t limit_ns, void* stream) {
 }
 
 int moe_profile_enable(int kernel_id) {
-  if (kernel_id < 0 || kernel_id > 11) return MOE_ERR_INVALID_ARG;
+  if (kernel_id < 0 || kernel_id > 12) return MOE_ERR_INVALID_ARG;
   std::lock_guard<std::mutex> lock(g_profile_mutex);
   g_profile_id.store(kernel_id, std::memory_order_relaxed);
   g_profile_n = 0;
@@ -473,7 +473,7 @@ namespace tcmoe {
 namespace {
 // Regions of the backward workspace, in order, each on a 1 KiB boundary.
 struct BwdPlan {
-  size_t status, poff, mt_prefix, mp_prefix, pair_prow, xs, dos, dh, h, da1, da3, dxs, total;
+  size_t status, poff, mt_prefix, mp_prefix, pair_prow, xs, dos, dh, h, da1, da3, dxs, g_row, dkey, wgt, total;
 };
 BwdPlan bwd_plan(const moe_shape_t& s) {
   BwdPlan p{};
@@ -497,6 +497,9 @@ BwdPlan bwd_plan(const moe_shape_t& s) {
   p.da1 = take(R * (size_t)s.f * 2);
   p.da3 = take(R * (size_t)s.f * 2);
   p.dxs = take(R * (size_t)s.d * 2);
+  p.g_row = take(R * 4);                       // moe_gate_backward: row dots, then key gradients per padded row
+  p.dkey = take(P * 4);                        //   key gradients per pair
+  p.wgt = take(E * (size_t)s.d * 4);           //   the gate weight transposed
   p.total = off;
   return p;
 }
@@ -554,6 +557,46 @@ int moe_layer_backward(const moe_shape_t* shape, const void* x, const void* dy, 
   a.dxs = at<void>(ws, p.dxs);
   a.status = at<int32_t>(ws, p.status);
   TCMOE_CUDA(launch_layer_backward(to_shape(*shape), a, static_cast<cudaStream_t>(stream)));
+  return MOE_OK;
+}
+
+int moe_gate_backward(const moe_shape_t* shape, const float* logits, const float* logit_bias, int64_t bias_row_stride,
+                      const int32_t* topk_idx, const float* topk_w, const moe_layout_t* layout, const float* w_gate,
+                      void* dx, float* dw_gate, void* ws, size_t ws_bytes, void* stream) {
+  int rc = check_shape(shape);
+  if (rc != MOE_OK) return rc;
+  if (shape->flags & ~MOE_FLAG_SPARSE_TOPK) return MOE_ERR_INVALID_ARG;
+  if (topk_idx == nullptr || topk_w == nullptr || w_gate == nullptr || dx == nullptr || dw_gate == nullptr ||
+      ws == nullptr)
+    return MOE_ERR_INVALID_ARG;
+  if (shape->score_fn == MOE_SCORE_SIGMOID && logits == nullptr) return MOE_ERR_INVALID_ARG;
+  if (logit_bias != nullptr && bias_row_stride != 0 && bias_row_stride != shape->E) return MOE_ERR_INVALID_ARG;
+  if ((rc = check_layout(layout)) != MOE_OK) return rc;
+  if (!aligned(dx, 128) || !aligned(ws, 128) || !aligned(w_gate, 16) || !aligned(dw_gate, 16) ||
+      !aligned(topk_idx, 16) || !aligned(topk_w, 16) || !aligned(logits, 16) || !aligned(logit_bias, 4))
+    return MOE_ERR_MISALIGNED;
+  const BwdPlan p = bwd_plan(*shape);
+  if (ws_bytes < p.total) return MOE_ERR_WORKSPACE_TOO_SMALL;
+  if (!have_device()) return MOE_ERR_CUDA;
+  GateBwdArgs a{};
+  a.topk_idx = topk_idx;
+  a.topk_w = topk_w;
+  a.expert_counts = layout->expert_counts;
+  a.logits = logits;
+  a.bias = logit_bias;
+  a.bias_stride = bias_row_stride;
+  a.w_gate = w_gate;
+  a.dx = dx;
+  a.dw_gate = dw_gate;
+  a.poff = at<int32_t>(ws, p.poff);
+  a.pair_prow = at<int32_t>(ws, p.pair_prow);
+  a.xs = at<void>(ws, p.xs);
+  a.h = at<void>(ws, p.h);
+  a.dh = at<void>(ws, p.dh);
+  a.g_row = at<float>(ws, p.g_row);
+  a.dkey = at<float>(ws, p.dkey);
+  a.wgt = at<float>(ws, p.wgt);
+  TCMOE_CUDA(launch_gate_backward(to_shape(*shape), a, static_cast<cudaStream_t>(stream)));
   return MOE_OK;
 }
 

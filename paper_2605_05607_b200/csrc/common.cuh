@@ -9,7 +9,7 @@ namespace tcmoe {
 // ---- status block at the start of the workspace (16 x int32) --------------------------------
 enum StatusSlot { ST_CODE = 0, ST_WHERE = 1, ST_DETAIL = 2, ST_AUX = 3, ST_ABORT = 4, ST_WARN = 5 };
 enum KernelId { KID_TOPK = 1, KID_MASKS = 2, KID_FILL = 3, KID_DISPATCH = 4, KID_GEMM1 = 5, KID_GEMM2 = 6,
-                KID_COMBINE = 7, KID_GATE = 8, KID_SELFTEST = 9, KID_WGRAD = 10, KID_BWD = 11 };
+                KID_COMBINE = 7, KID_GATE = 8, KID_SELFTEST = 9, KID_WGRAD = 10, KID_BWD = 11, KID_GATE_BWD = 12 };
 constexpr int DEV_TIMEOUT = 1;
 constexpr int DEV_INDEX_OUT_OF_RANGE = 2;
 constexpr int WARN_NONFINITE_LOGIT = 1;
@@ -121,6 +121,24 @@ struct BwdArgs {
 };
 size_t bwd_row_capacity(const Shape& s);
 cudaError_t launch_layer_backward(const Shape& s, const BwdArgs& a, cudaStream_t st);
+// gate_bwd.cu: gradient of the gate network, after launch_layer_backward on the same scratch
+struct GateBwdArgs {
+  const int32_t* topk_idx;          // [T, k]
+  const float* topk_w;              // [T, k]
+  const int32_t* expert_counts;     // [E] (the forward layout)
+  const float* logits;              // [T, E] fp32 router logits of the forward (sigmoid scores only, else may be NULL)
+  const float* bias;                // NULL, [E] (stride 0) or [T, E] (stride E)
+  int64_t bias_stride;
+  const float* w_gate;              // [d, E] fp32
+  void* dx;                         // [T, d] bf16, in / out: the gate path is added
+  float* dw_gate;                   // [d, E] fp32 out
+  // left behind by launch_layer_backward
+  const int32_t *poff, *pair_prow;
+  const void *xs, *h, *dh;
+  // scratch
+  float *g_row, *dkey, *wgt;        // [bwd_row_capacity], [T * k], [E, d]
+};
+cudaError_t launch_gate_backward(const Shape& s, const GateBwdArgs& a, cudaStream_t st);
 // ffn.cu
 struct FfnArgs {
   const void* a_src;          // GEMM-1 activations: xg (gather_div = 1) or x (gather_div = k)

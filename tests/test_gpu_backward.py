@@ -135,3 +135,111 @@ def test_backward_fullsize_sampled(name):
     toks = synth.sample_tokens(cfg, 96)[::4][:24]
     dx_ref, _ = O.layer_backward(xb[toks], idx[toks], w[toks], w1, w3, w2, dy[toks])
     close(O.bf16_to_f64(H.bf16_host(bw.dx[torch.from_numpy(toks).cuda()])), dx_ref, f"{name} dx")
+
+
+GATE_CASES = SMALL + [
+    synth.MoEConfig("sigmoid-locality", T=260, d=192, f=256, E=16, k=4, G=4, score_fn=1, bias="locality", seed=21),
+    synth.MoEConfig("softmax-zipf-k8", T=200, d=256, f=128, E=32, k=8, G=8, bias="zipf", zipf_s=1.1, seed=22),
+]
+
+
+def _gate_backward(bw):
+    run, cfg = bw.run, bw.cfg
+    dwg = torch.full((cfg.d, cfg.E), 7.0, dtype=torch.float32, device="cuda")
+    B.moe_gate_backward(run.shape, run.logits, run.t["bias"], run.idx, run.w, run.lay, run.t["w_gate"], bw.dx, dwg, bw.ws)
+    torch.cuda.synchronize()
+    st = B.moe_status(bw.ws)
+    assert st[0] == 0 and st[4] == 0, f"device status {st}"
+    return dwg
+
+
+@pytest.mark.parametrize("cfg", GATE_CASES, ids=lambda c: c.name)
+def test_gate_backward_matches_oracle(cfg):
+    """moe_layer_backward followed by moe_gate_backward: dw_gate against the oracle's gate gradient, the total dx
+    against expert path + gate path; softmax and sigmoid scores, no bias / per-expert bias / per-token bias."""
+    bw = Backward(cfg)
+    bw()
+    run = bw.run
+    dx_experts = bw.dx.clone()
+    dwg = _gate_backward(bw)
+    xb = H.bf16_host(run.t["x"])
+    dy = O.bf16_to_f64(H.bf16_host(bw.dy))[: cfg.T]
+    idx, w = run.host_idx(), run.host_w()
+    w1, w3, w2 = (H.bf16_host(run.t[n]) for n in ("w1", "w3", "w2"))
+    wg = run.t["w_gate"].cpu().numpy()
+    dwg_ref, dxg_ref, dkey_ref, _ = O.gate_backward(xb, wg, run.host_bias(), idx, cfg.score_fn, w1, w3, w2, dy)
+    got = dwg.cpu().numpy().astype(np.float64)
+    if cfg.k == 1:
+        # a single selected expert has weight 1 whatever its key: nothing reaches the gate, exactly
+        assert not got.any() and torch.equal(bw.dx, dx_experts)
+        assert np.abs(dwg_ref).max() <= 1e-12
+        return
+    if cfg.T >= 16:
+        close(got, dwg_ref, "dw_gate")
+    else:
+        # one token: every entry of dw_gate carries the same two key gradients, so nothing averages out and the
+        # mean error IS the error of one bf16-rounded dot product; only the max bar applies
+        mx, _ = H.out_errors(got, dwg_ref)
+        assert mx <= MAX_REL, f"dw_gate: max rel {mx:.3e}"
+    dx_ref, _ = O.layer_backward(xb, idx, w, w1, w3, w2, dy)
+    close(O.bf16_to_f64(H.bf16_host(bw.dx))[: cfg.T], dx_ref + dxg_ref, "dx with the gate path")
+    # the gate path by itself: what the call added to dx (bf16 roundings of both sides allowed for)
+    added = O.bf16_to_f64(H.bf16_host(bw.dx))[: cfg.T] - O.bf16_to_f64(H.bf16_host(dx_experts))[: cfg.T]
+    tol = 2.0 ** -7 * np.abs(dx_ref + dxg_ref) + 2e-2 * np.abs(dxg_ref).max()
+    assert np.all(np.abs(added - dxg_ref) <= tol), "gate path of dx"
+    # columns of experts nobody selected are exact zeros
+    unused = np.setdiff1d(np.arange(cfg.E), np.unique(idx))
+    assert not got[:, unused].any()
+    # deterministic: the whole backward again gives the same bits
+    keep = (bw.dx.clone(), dwg.clone())
+    bw()
+    dwg2 = _gate_backward(bw)
+    assert torch.equal(keep[0], bw.dx) and torch.equal(keep[1], dwg2)
+
+
+def test_gate_backward_argument_checks():
+    cfg = synth.MoEConfig("sig", T=64, d=64, f=64, E=8, k=2, G=2, score_fn=1, seed=5)
+    bw = Backward(cfg)
+    bw()
+    run = bw.run
+    dwg = torch.zeros(cfg.d, cfg.E, dtype=torch.float32, device="cuda")
+    with pytest.raises(B.MoEError) as ei:      # sigmoid scores need the forward's logits
+        B.moe_gate_backward(run.shape, None, run.t["bias"], run.idx, run.w, run.lay, run.t["w_gate"], bw.dx, dwg, bw.ws)
+    assert ei.value.code == B.MOE_ERR_INVALID_ARG
+    with pytest.raises(B.MoEError) as ei:
+        B.moe_gate_backward(run.shape, run.logits, run.t["bias"], run.idx, run.w, run.lay, run.t["w_gate"], bw.dx, dwg,
+                            bw.ws[:4096])
+    assert ei.value.code == B.MOE_ERR_WORKSPACE_TOO_SMALL
+
+
+def test_gate_backward_fullsize_sampled():
+    """C4 at full size (per-token locality bias, softmax): the dw_gate columns of four experts in full and the total dx
+    on 16 sampled tokens.  The oracle needs dL/dw of every pair of the sampled experts / tokens only."""
+    cfg = synth.ALL_CONFIGS["C4"]
+    bw = Backward(cfg)
+    bw()
+    run = bw.run
+    dwg = _gate_backward(bw)
+    idx, w = run.host_idx(), run.host_w()
+    xb = H.bf16_host(run.t["x"])
+    dy = O.bf16_to_f64(H.bf16_host(bw.dy))
+    wg = run.t["w_gate"].cpu().numpy()
+    bias = run.host_bias()
+    w1, w3, w2 = Slabs(run.t["w1"]), Slabs(run.t["w3"]), Slabs(run.t["w2"])
+    # tokens: a sample for dx, plus every token of two lightly loaded experts for their dw_gate columns
+    counts = np.bincount(idx.reshape(-1), minlength=cfg.E)
+    picks = [int(e) for e in np.argsort(counts)[:2]]
+    toks = synth.sample_tokens(cfg, 64)[::4][:16]
+    need = np.unique(np.concatenate([toks] + [np.nonzero((idx == e).any(axis=1))[0] for e in picks]))
+    b = None if bias is None else (bias if bias.ndim == 1 else bias[need])
+    _, dxg, dkey, _ = O.gate_backward(xb[need], wg, b, idx[need], cfg.score_fn, w1, w3, w2, dy[need])
+    x64 = O.bf16_to_f64(xb[need])
+    got = dwg.cpu().numpy().astype(np.float64)
+    for e in picks:
+        col = np.zeros(cfg.d)
+        hit_t, hit_j = np.nonzero(idx[need] == e)
+        col = (dkey[hit_t, hit_j][:, None] * x64[hit_t]).sum(axis=0)
+        close(got[:, e], col, f"dw_gate[:, {e}]")
+    pos = np.searchsorted(need, toks)
+    dx_ref, _ = O.layer_backward(xb[toks], idx[toks], w[toks], w1, w3, w2, dy[toks])
+    close(O.bf16_to_f64(H.bf16_host(bw.dx[torch.from_numpy(toks).cuda()])), dx_ref + dxg[pos], "C4 dx with the gate path")

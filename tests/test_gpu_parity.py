@@ -390,6 +390,9 @@ def test_no_entry_point_writes_outside_its_buffers(cfg):
         g["d" + n] = Guarded(t[n].numel(), torch.bfloat16)
     B.moe_layer_backward(shape, t["x"], y, g["idx"].t, g["w"].t, lay, t["w1"], t["w3"], t["w2"], g["dx"].t.view(-1, d),
                          g["dw1"].t.view_as(t["w1"]), g["dw3"].t.view_as(t["w3"]), g["dw2"].t.view_as(t["w2"]), g["bws"].t)
+    g["dw_gate"] = Guarded(d * E, torch.float32)
+    B.moe_gate_backward(shape, g["logits"].t, t["bias"], g["idx"].t, g["w"].t, lay, t["w_gate"], g["dx"].t.view(-1, d),
+                        g["dw_gate"].t.view(d, E), g["bws"].t)
     if cfg.d % 16 == 0 and cfg.f % 16 == 0:
         wq = {n: Guarded(t[n].numel(), torch.uint8) for n in ("w1", "w3", "w2")}
         sc = {n: Guarded(E * t[n].shape[2], torch.float32) for n in ("w1", "w3", "w2")}
