@@ -109,9 +109,10 @@ class Slabs:
         return synth.bf16_bits(self.w[int(e)])
 
 
-@pytest.mark.parametrize("name", ["C3", "C4"])
+@pytest.mark.parametrize("name", ["C3", "C4", "C5a"])
 def test_backward_fullsize_sampled(name):
-    """Full size (C4: 131 072 expert rows; C3: Zipf-skewed with empty and tiny experts): weight gradients of the most
+    """Full size (C4: 131 072 expert rows; C3: Zipf-skewed with empty and tiny experts; C5a: the benchmark's workload,
+    262 144 expert rows, 22.5 GB of weights and as much of gradients): weight gradients of the most
     loaded, the least loaded and two more experts in full, dx on 24 sampled tokens."""
     cfg = synth.ALL_CONFIGS[name]
     bw = Backward(cfg)
