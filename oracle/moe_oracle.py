@@ -316,7 +316,8 @@ def layer_backward(x_bits: np.ndarray, topk_idx: np.ndarray, topk_w: np.ndarray,
     the gradients of  L = sum(dy * y)  are
         dx[t]  = sum_j  w[t, j] * dFFN/da (x[t]) applied to dy[t]
         dW*[e] = sum over the pairs (t, j) with idx[t, j] = e  of  w[t, j] * (their expert-level gradient).
-    ``dy`` float64 [T, d]; ``topk_w`` [T, k].  With ``experts`` only those experts' weight gradients are formed
+    ``dy`` float64 [T, d]; ``topk_w`` [T, k]; entries of ``topk_idx`` below 0 are slots not in use and contribute
+    nothing.  With ``experts`` only those experts' weight gradients are formed
     (dx is then omitted).  Returns (dx [T, d] or None, {e: (dW1, dW3, dW2)}), all float64."""
     idx = np.asarray(topk_idx, dtype=np.int64)
     w = np.asarray(topk_w, dtype=np.float64)
@@ -324,6 +325,8 @@ def layer_backward(x_bits: np.ndarray, topk_idx: np.ndarray, topk_w: np.ndarray,
     dx = np.zeros((T, x_bits.shape[1]), dtype=np.float64) if experts is None else None
     grads = {}
     for e in (np.unique(idx) if experts is None else experts):
+        if e < 0:            # slot not in use (a routing table trimmed to one group's experts, Sec. III-D)
+            continue
         hit_t, hit_j = np.nonzero(idx == e)
         w1, w3, w2 = bf16_to_f64(w1_bits[e]), bf16_to_f64(w3_bits[e]), bf16_to_f64(w2_bits[e])
         if hit_t.size == 0:

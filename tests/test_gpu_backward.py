@@ -244,3 +244,40 @@ def test_gate_backward_fullsize_sampled():
     pos = np.searchsorted(need, toks)
     dx_ref, _ = O.layer_backward(xb[toks], idx[toks], w[toks], w1, w3, w2, dy[toks])
     close(O.bf16_to_f64(H.bf16_host(bw.dx[torch.from_numpy(toks).cuda()])), dx_ref + dxg[pos], "C4 dx with the gate path")
+
+
+def test_backward_on_a_sparse_routing_table():
+    """MOE_FLAG_SPARSE_TOPK (slots of topk_idx may be -1, one token without any slot): dx and the weight gradients
+    against the oracle restricted to the slots in use; the token without slots gets a zero row of dx."""
+    cfg = synth.MoEConfig("sparse-bwd", T=300, d=128, f=192, E=12, k=4, G=3, seed=21)
+    run = H.Run(cfg, B.MOE_FLAG_SPARSE_TOPK)
+    run.route()
+    rng = np.random.default_rng(3)
+    idx = run.host_idx().copy()
+    drop = rng.random(idx.shape) < 0.4
+    drop[5] = True
+    drop[6] = False
+    idx[drop] = -1
+    run.idx[: cfg.P] = torch.from_numpy(idx.reshape(-1)).cuda()
+    run.dispatch()
+    g = torch.Generator(device="cuda")
+    g.manual_seed(5)
+    dy = torch.randn(cfg.T, cfg.d, generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    dx = torch.full((cfg.T, cfg.d), 7.0, dtype=torch.bfloat16, device="cuda")
+    dw = {n: torch.full_like(run.t[n], 7.0) for n in ("w1", "w3", "w2")}
+    ws = torch.zeros(B.moe_backward_workspace_bytes(run.shape), dtype=torch.uint8, device="cuda")
+    B.moe_layer_backward(run.shape, run.t["x"], dy, run.idx, run.w, run.lay, run.t["w1"], run.t["w3"], run.t["w2"], dx,
+                         dw["w1"], dw["w3"], dw["w2"], ws)
+    torch.cuda.synchronize()
+    assert B.moe_status(ws)[0] == 0
+    w1, w3, w2 = (H.bf16_host(run.t[n]) for n in ("w1", "w3", "w2"))
+    dx_ref, grads = O.layer_backward(H.bf16_host(run.t["x"]), idx, run.host_w(), w1, w3, w2,
+                                     O.bf16_to_f64(H.bf16_host(dy)))
+    got = O.bf16_to_f64(H.bf16_host(dx))
+    close(got, dx_ref, "sparse dx")
+    assert not got[5].any() and not dx_ref[5].any()
+    for n, pos in (("w1", 0), ("w3", 1), ("w2", 2)):
+        ref = np.zeros(tuple(run.t[n].shape))
+        for e, gr in grads.items():
+            ref[e] = gr[pos]
+        close(O.bf16_to_f64(H.bf16_host(dw[n])), ref, f"sparse d{n}")

@@ -683,3 +683,24 @@ def test_gate_backward_special_cases():
     assert np.abs(dkey.sum(axis=1)).max() <= 1e-14 * np.abs(dkey).max()
     dwg2, dxg2, _, _ = O.gate_backward(xb, wg, bias, idx, O.SCORE_SOFTMAX, w1b, w3b, w2b, 3.0 * dy)
     assert np.allclose(dwg2, 3.0 * dwg, rtol=1e-13, atol=0) and np.allclose(dxg2, 3.0 * dxg, rtol=1e-13, atol=0)
+
+
+def test_layer_backward_ignores_slots_not_in_use():
+    """A slot of topk_idx below 0 contributes nothing: the same result as pointing the slot at any expert with gate
+    weight 0 (whose contribution is w * (...) = 0 term by term)."""
+    rng = np.random.default_rng(41)
+    T, d, f, E, k = 5, 6, 4, 3, 2
+    xb = O.f64_to_bf16_bits(rng.standard_normal((T, d)))
+    w1b, w3b, w2b = (O.f64_to_bf16_bits(rng.standard_normal(s) * 0.4) for s in ((E, d, f), (E, d, f), (E, f, d)))
+    idx = np.array([[0, 1], [1, -1], [2, 0], [-1, -1], [1, 2]], dtype=np.int32)
+    w = rng.uniform(0.2, 0.8, size=(T, k))
+    dy = rng.standard_normal((T, d))
+    dx, grads = O.layer_backward(xb, idx, w, w1b, w3b, w2b, dy)
+    idx2, w2 = idx.copy(), w.copy()
+    w2[idx < 0] = 0.0
+    idx2[idx < 0] = 2
+    dx2, grads2 = O.layer_backward(xb, idx2, w2, w1b, w3b, w2b, dy)
+    assert np.allclose(dx, dx2, rtol=0, atol=1e-15) and not dx[3].any()
+    for e in range(E):
+        for a, b in zip(grads[e], grads2[e]):
+            assert np.allclose(a, b, rtol=0, atol=1e-15)
