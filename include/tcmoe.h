@@ -219,8 +219,8 @@ int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, co
 
 /* ---- backward pass ----------------------------------------------------------------------------------
  * Sec. VI-A evaluates training, forward + backward, of the layer of Sec. II-A.  For FIXED routing (expert indices
- * and gate weights as the forward produced them, held constant: the gate network's own gradient is not part of
- * this call), with dy = dL/dy:
+ * and gate weights as the forward produced them, held constant: the gate network's own gradient is the separate
+ * call moe_gate_backward below), with dy = dL/dy:
  *     dx[t]  = sum_j w[t,j] * dFFN_e/da (x[t]) applied to dy[t]          [T, d] bf16
  *     dw1[e] = Xs_e^T dA1_e,  dw3[e] = Xs_e^T dA3_e,  dw2[e] = H_e^T dO_e   [E, d, f], [E, d, f], [E, f, d] bf16
  * where Xs_e / H_e / dO_e / dA*_e are the rows of expert e (dO = w * dy, dH = dO W2^T, dA1 = dH * a3 * silu'(a1),
@@ -230,7 +230,8 @@ int moe_layer_host(const moe_shape_t* shape, const void* x_host, void* x_dev, co
  *   topk_idx, topk_w, layout   as written by moe_layer / moe_route + moe_dispatch for the same x
  *   w1, w3, w2  the forward weights, read in place (transposed operands are read K-major, nothing is repacked)
  *   ws          moe_backward_workspace_bytes(shape) bytes, 128-byte aligned, status block at its start (zero it
- *               once or call moe_status_reset; read with moe_status)
+ *               once or call moe_status_reset; read with moe_status); the size includes the scratch of
+ *               moe_gate_backward, which reads what this call leaves there
  * shape->flags: 0 or MOE_FLAG_SPARSE_TOPK. */
 int moe_backward_workspace_bytes(const moe_shape_t* shape, size_t* bytes);
 int moe_layer_backward(const moe_shape_t* shape, const void* x, const void* dy, const int32_t* topk_idx,
