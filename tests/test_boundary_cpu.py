@@ -127,9 +127,26 @@ def test_argument_checks_happen_before_any_device_work(lib):
     # null layout
     assert B.lib().moe_dispatch(ctypes.byref(shape), None, i32.data_ptr(), None, None, ws_al.data_ptr(), n,
                                 None) == B.MOE_ERR_INVALID_ARG
+    # gate gradient: sigmoid scores need the forward's logits; a short backward workspace is refused
+    lay = B.Layout(**{k: torch.zeros(64, dtype=torch.int32) for k in ("expert_counts", "expert_offsets", "group_counts",
+                                                                      "group_offsets", "pair_row", "row_pair", "al",
+                                                                      "disp_token", "row_src")})
+    nb = B.moe_backward_workspace_bytes(shape)
+    bws = torch.zeros(nb + 256, dtype=torch.uint8)
+    bws_al = bws[(-bws.data_ptr()) % 128:][:nb]
+    dxb = torch.zeros(cfg.T * cfg.d * 2 + 256, dtype=torch.uint8)
+    dx = dxb[(-dxb.data_ptr()) % 128:][: cfg.T * cfg.d * 2]
+    wg = torch.zeros(cfg.d * cfg.E, dtype=torch.float32)
+    sig = B.make_shape(cfg.with_(score_fn=1))
+    assert rc(lambda: B.moe_gate_backward(sig, None, None, i32, w, lay, wg, dx, wg.clone(), bws_al)) == B.MOE_ERR_INVALID_ARG
+    assert rc(lambda: B.moe_gate_backward(shape, None, None, i32, w, lay, wg, dx, wg.clone(), bws_al[:4096])) \
+        == B.MOE_ERR_WORKSPACE_TOO_SMALL
+    assert rc(lambda: B.moe_gate_backward(B.make_shape(cfg, B.MOE_FLAG_FUSED_FFN), None, None, i32, w, lay, wg, dx,
+                                          wg.clone(), bws_al)) == B.MOE_ERR_INVALID_ARG
     if not torch.cuda.is_available():
         assert rc(lambda: B.moe_route(shape, None, None, None, f32, i32, w, ws_al)) == B.MOE_ERR_CUDA
         assert rc(lambda: B.moe_status(ws_al)) == B.MOE_ERR_CUDA
+        assert rc(lambda: B.moe_gate_backward(shape, None, None, i32, w, lay, wg, dx, wg.clone(), bws_al)) == B.MOE_ERR_CUDA
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
